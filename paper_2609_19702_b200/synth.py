@@ -1,0 +1,214 @@
+"""Seeded synthetic decode-attention workloads.
+
+This module only DRAWS INPUTS: random tensors with the shapes, value distributions and position
+mixes of the five benchmark configurations, block tables, and valid skip traces.  It holds none
+of the method's arithmetic (no mask, no attention), so both the CUDA binding and the CPU oracle
+can be fed from it without sharing anything else.
+
+Everything is generated on the host with ``numpy.random.default_rng(seed)`` and rounded to
+bfloat16 (stored as uint16 bit patterns); the very same arrays go to the GPU and to the oracle,
+so input rounding is not part of any error budget.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+from typing import Dict, Optional
+
+import numpy as np
+
+BF16_NAN = np.uint16(0x7FC0)
+BASE_SEED = 19702
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (nearest even); returns the uint16 bit patterns."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    bits = x.view(np.uint32)
+    rounded = (bits + np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    return rounded.astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+@dataclass(frozen=True)
+class Workload:
+    """One benchmark configuration (shapes follow the token counts of the paper's Table 1)."""
+    name: str
+    index: int                 # 1..5, seeds the generator
+    batch: int
+    num_q_heads: int
+    num_kv_heads: int
+    head_dim: int
+    prompt_len: int            # L_p
+    grid_h: int
+    grid_w: int
+    row_extra: int             # row-end / separator tokens per image row (0 or 1)
+    window: int                # N_r
+    n_att: int                 # N_att
+    pos_lo: int                # decode position p drawn uniformly from [pos_lo, pos_hi]
+    pos_hi: int
+    positional: bool = False   # add 0.5 x a 2-D sin-cos embedding to image-token q/k/v
+    paged: bool = False
+    block_size: int = 16
+    share_cache: bool = False  # all requests read one cache (batch stride 0); positions 1..batch
+
+    @property
+    def stride(self) -> int:   # tokens per image row in raster order
+        return self.grid_w + self.row_extra
+
+    @property
+    def image_tokens(self) -> int:
+        return self.grid_h * self.stride
+
+    @property
+    def max_seq_len(self) -> int:
+        return self.prompt_len + self.image_tokens
+
+
+def workload(index: int, batch: Optional[int] = None, window: Optional[int] = None,
+             n_att: Optional[int] = None) -> Workload:
+    """The five configurations.  N_att is 5 % of the image tokens (95 % sparsity) unless given."""
+    table = {
+        1: Workload("tiny", 1, 256, 8, 8, 64, 32, 16, 16, 0, 64, 13, 1, 256, share_cache=True),
+        2: Workload("mid_mha", 2, 32, 20, 20, 64, 120, 32, 32, 0, 256, 52, 1, 1024, positional=True),
+        3: Workload("mha_7b", 3, 64, 32, 32, 128, 600, 24, 24, 0, 128, 29, 289, 576),
+        4: Workload("gqa_long", 4, 8, 32, 8, 128, 64, 90, 90, 1, 1024, 410, 4096, 8190, positional=True),
+        5: Workload("paged_sweep", 5, 256, 32, 32, 128, 200, 64, 64, 1, 512, 208, 1, 4160, paged=True),
+    }
+    w = table[index]
+    if batch is not None:
+        w = replace(w, batch=batch)
+    if window is not None:
+        w = replace(w, window=window)
+    if n_att is not None:
+        w = replace(w, n_att=n_att)
+    return w
+
+
+def _positional(w: Workload) -> np.ndarray:
+    """[image_tokens, D] float32: textbook 2-D sin-cos embedding, rows from r, columns from c."""
+    d = w.head_dim
+    half = d // 2
+    tok = np.arange(w.image_tokens)
+    r = (tok // w.stride).astype(np.float64)
+    c = (tok % w.stride).astype(np.float64)
+    is_grid = (tok % w.stride) < w.grid_w
+    i = np.arange(half // 2, dtype=np.float64)
+    freq = 10000.0 ** (-2.0 * i / half)
+    emb = np.zeros((w.image_tokens, d), dtype=np.float64)
+    emb[:, 0:half:2] = np.sin(r[:, None] * freq[None, :])
+    emb[:, 1:half:2] = np.cos(r[:, None] * freq[None, :])
+    emb[:, half::2] = np.sin(c[:, None] * freq[None, :])
+    emb[:, half + 1::2] = np.cos(c[:, None] * freq[None, :])
+    emb[~is_grid] = 0.0
+    return (0.5 * emb).astype(np.float32)
+
+
+def random_valid_trace(rng: np.random.Generator, window: int, n_att: int, shape=()) -> np.ndarray:
+    """Random skip traces [..., window - n_att]: entry k (0-based) is an offset in
+    [0, n_att - 1 + k] that no earlier entry used -- the only constraint a trace must meet."""
+    m = window - n_att
+    n = int(np.prod(shape)) if shape else 1
+    out = np.zeros((n, max(m, 0)), dtype=np.int32)
+    for i in range(n):
+        used = np.zeros(window, dtype=bool)
+        for k in range(m):
+            free = np.flatnonzero(~used[: n_att + k])
+            o = int(free[rng.integers(len(free))])
+            used[o] = True
+            out[i, k] = o
+    return out.reshape(tuple(shape) + (max(m, 0),))
+
+
+def make_inputs(w: Workload, seed: Optional[int] = None, poison: bool = True) -> Dict[str, object]:
+    """Draw one batch of inputs for workload ``w`` on the host.
+
+    Returns a dict with
+      q            uint16 [B, H_q, D]   bf16 bits
+      k_cache/v_cache uint16, flat view of  [B, S_max, H_kv, D]  (contiguous)  or
+                                            [num_blocks, block_size, H_kv, D]  (paged)
+      strides      (stride_b_or_block, stride_token, stride_head) in elements
+      seq_len, prompt_len  int32 [B];  position int32 [B] (= seq_len - prompt_len)
+      block_table  int32 [B, max_blocks] or None;  block_size
+    Cache rows at positions >= seq_len are NaN when ``poison`` (never for a shared cache).
+    """
+    rng = np.random.default_rng(BASE_SEED + w.index if seed is None else seed)
+    b, hq, hkv, d = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    s_max = w.max_seq_len
+    pos_emb = _positional(w) if w.positional else None
+
+    if w.share_cache:
+        position = (np.arange(b, dtype=np.int32) % w.image_tokens) + 1
+    else:
+        position = rng.integers(w.pos_lo, w.pos_hi + 1, size=b, dtype=np.int32)
+    prompt_len = np.full(b, w.prompt_len, dtype=np.int32)
+    seq_len = prompt_len + position
+
+    q = rng.standard_normal((b, hq, d), dtype=np.float32)
+    if pos_emb is not None:
+        q += pos_emb[position - 1][:, None, :]
+    q_bits = f32_to_bf16_bits(q)
+
+    def draw_seq() -> np.ndarray:
+        x = rng.standard_normal((s_max, hkv, d), dtype=np.float32)
+        if pos_emb is not None:
+            x[w.prompt_len:] += pos_emb[:, None, :]
+        return f32_to_bf16_bits(x)
+
+    row = hkv * d
+    block_table = None
+    if w.paged:
+        bs = w.block_size
+        max_blocks = (s_max + bs - 1) // bs
+        num_blocks = b * max_blocks
+        block_table = rng.permutation(num_blocks).astype(np.int32).reshape(b, max_blocks)
+        k_cache = np.empty((num_blocks, bs, hkv, d), dtype=np.uint16)
+        v_cache = np.empty((num_blocks, bs, hkv, d), dtype=np.uint16)
+        pad = max_blocks * bs - s_max
+        for i in range(b):
+            for cache in (k_cache, v_cache):
+                x = draw_seq()
+                if poison:
+                    x[seq_len[i]:] = BF16_NAN
+                if pad:
+                    x = np.concatenate([x, np.full((pad, hkv, d), BF16_NAN, dtype=np.uint16)])
+                cache[block_table[i]] = x.reshape(max_blocks, bs, hkv, d)
+        strides = (bs * row, row, d)
+    elif w.share_cache:
+        k_cache = draw_seq().reshape(1, s_max, hkv, d)
+        v_cache = draw_seq().reshape(1, s_max, hkv, d)
+        strides = (0, row, d)
+    else:
+        k_cache = np.empty((b, s_max, hkv, d), dtype=np.uint16)
+        v_cache = np.empty((b, s_max, hkv, d), dtype=np.uint16)
+        for i in range(b):
+            for cache in (k_cache, v_cache):
+                x = draw_seq()
+                if poison:
+                    x[seq_len[i]:] = BF16_NAN
+                cache[i] = x
+        strides = (s_max * row, row, d)
+
+    return {
+        "workload": w,
+        "q": q_bits,
+        "k_cache": k_cache.reshape(-1),
+        "v_cache": v_cache.reshape(-1),
+        "cache_shape": k_cache.shape,
+        "strides": strides,
+        "seq_len": seq_len.astype(np.int32),
+        "prompt_len": prompt_len,
+        "position": position.astype(np.int32),
+        "block_table": block_table,
+        "block_size": w.block_size if w.paged else 0,
+        "max_seq_len": s_max,
+    }
+
+
+def shard_requests(batch: int, world_size: int, rank: int) -> range:
+    """Contiguous slice of request ids owned by ``rank`` (requests are independent units)."""
+    base, extra = divmod(batch, world_size)
+    lo = rank * base + min(rank, extra)
+    return range(lo, lo + base + (1 if rank < extra else 0))
