@@ -1,0 +1,207 @@
+/*
+ * dsa.h -- C ABI of the diagonal-aware sparse decode-attention library for NVIDIA B200 (sm_100a).
+ *
+ * One call = one decode step of one transformer layer: every request of a batch has ONE query
+ * token per head and attends over its KV cache.  The sparse call keeps the whole prompt and,
+ * inside a recent window of the decode (image) tokens, drops the keys that lie on the skipped
+ * diagonals -- keys at fixed distances behind the query -- so that dropped keys are never read
+ * from memory.  (Paper: "Understanding and Exploiting Diagonal Attention Sparsity in
+ * Autoregressive Image Generation", Section 4 and Algorithm 1.)
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; it must stay valid until the
+ *     work queued on `stream` has finished.  The dsa_problem / dsa_diag_params structs themselves
+ *     are HOST memory, read during the call only.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream);
+ *     the library never synchronises, allocates no device memory and keeps no state between
+ *     calls.  Scratch comes from the caller's `workspace` (device, 256-byte aligned), sized by
+ *     dsa_workspace_size(); it may be reused by the next call on the same stream.
+ *   - Arguments are checked on the host before anything is launched.  Values that live in
+ *     device memory (seq_len, prompt_len, block ids, skip offsets) cannot be checked there;
+ *     kernels clamp them into range instead, so bad values give wrong numbers, not faults.
+ *   - Return value: DSA_OK or a negative dsa_status.  After DSA_ERR_CUDA the CUDA error code is
+ *     available from dsa_last_cuda_error().
+ *   - There is no CPU path: without a CUDA device every compute call fails with DSA_ERR_CUDA.
+ *
+ * Positions.  For request b, prompt_len[b] = L_p tokens of prompt come first in the cache and
+ * are always attended.  p = seq_len[b] - prompt_len[b] decode tokens follow, the last of which
+ * is the token being decoded (its K/V are already in the cache); Algorithm 1's 0-based step is
+ * t = p - 1.  A key at cache position s >= L_p lies o = seq_len - 1 - s tokens behind the query.
+ */
+#ifndef DSA_H
+#define DSA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DSA_VERSION 100
+
+/* exported symbols (the library is built with hidden visibility for everything else) */
+#if defined(__GNUC__)
+#define DSA_API __attribute__((visibility("default")))
+#else
+#define DSA_API
+#endif
+
+typedef enum dsa_status {
+    DSA_OK = 0,
+    DSA_ERR_INVALID_ARG = -1,         /* null pointer, bad size, bad stride, N_att > window ...   */
+    DSA_ERR_UNSUPPORTED = -2,         /* head_dim not 64/128, group size not 1/2/4/8, window too   */
+                                      /* large for a LIST mask, ...                                */
+    DSA_ERR_WORKSPACE_TOO_SMALL = -3,
+    DSA_ERR_CUDA = -4                 /* a CUDA runtime call failed; see dsa_last_cuda_error()     */
+} dsa_status;
+
+typedef enum dsa_dtype { DSA_BF16 = 0, DSA_F32 = 1 } dsa_dtype;
+
+typedef enum dsa_mask_mode {
+    DSA_MASK_WINDOW = 0,  /* prompt + the `window` most recent decode tokens, nothing skipped      */
+    DSA_MASK_GRID = 1,    /* skipped diagonals derived from the raster grid (see dsa_diag_params)  */
+    DSA_MASK_LIST = 2     /* skipped diagonals given per head as a list of distances               */
+} dsa_mask_mode;
+
+/*
+ * The attention problem (inputs of Algorithm 1: the prompt KV cache K_p,V_p and the decode KV
+ * cache K,V, stored back to back per request, plus the query of the current step).
+ */
+typedef struct dsa_problem {
+    int32_t batch;             /* B, number of requests (>= 0)                                     */
+    int32_t num_q_heads;       /* H_q                                                              */
+    int32_t num_kv_heads;      /* H_kv; H_q / H_kv must be 1, 2, 4 or 8.  Query head h reads kv    */
+                               /* head h / (H_q / H_kv)                                            */
+    int32_t head_dim;          /* D: 64 or 128                                                     */
+    int32_t dtype;             /* dsa_dtype of q, k_cache, v_cache and out                         */
+    float sm_scale;            /* logit scale; 0 means 1/sqrt(D)                                   */
+    const void *q;             /* [B, H_q, D] contiguous                                           */
+    const void *k_cache;       /* keys;   rows of D contiguous elements, 16-byte aligned           */
+    const void *v_cache;       /* values; same layout and strides as k_cache                       */
+    /* Element strides.  Contiguous cache (block_table == NULL): token s of request b, kv head g
+     * starts at b*stride_batch + s*stride_token + g*stride_head (stride_batch may be 0 to let all
+     * requests read one cache).  Paged cache: token s lives in block
+     * id = block_table[b*max_blocks + s/block_size] at
+     * id*stride_batch + (s % block_size)*stride_token + g*stride_head.
+     * All strides must be multiples of 16 bytes. */
+    int64_t stride_batch;
+    int64_t stride_token;
+    int64_t stride_head;
+    const int32_t *seq_len;    /* [B] tokens in the cache, prompt included                         */
+    const int32_t *prompt_len; /* [B] L_p; values above seq_len[b] are read as seq_len[b]          */
+    const int32_t *block_table;/* [B, max_blocks] or NULL                                          */
+    int32_t max_blocks;        /* row length of block_table                                        */
+    int32_t block_size;        /* tokens per block (> 0 when paged)                                */
+    int32_t num_blocks;        /* blocks in the pool; block ids are clamped to [0, num_blocks)     */
+    int32_t max_seq_len;       /* HOST upper bound of seq_len[b]; sizes the launch.  Longer        */
+                               /* sequences are read as if they ended there                        */
+    int32_t max_prompt_len;    /* HOST upper bound of prompt_len[b], or 0 if unknown (the sparse   */
+                               /* call then plans for max_seq_len kept tokens)                     */
+    int32_t split_tokens;      /* kept tokens handled by one thread block; 0 = library chooses.    */
+                               /* Rounded up to the tile size, at most 1024                        */
+} dsa_problem;
+
+/*
+ * Which decode keys are kept (Algorithm 1 with its data-dependent selection made an input).
+ *
+ * With t = p - 1, the window holds the distances o = 0 .. min(t, window - 1) (the `window` = N_r
+ * most recent decode tokens, the current one included).  m = window - n_att diagonals are
+ * skipped in steady state.  Algorithm 1 selects them one per step from step n_att - 1 on, and an
+ * entry selected at step s is skipped from step s + 1 on; so at step t the first
+ * n_act = clamp(t - (n_att - 1), 0, m) selected distances are skipped.  A key chosen at step s
+ * with cache index j keeps the distance s - j at every later step (the "+1" shift of skip_idx).
+ *
+ *   LIST  skip_offsets[b][mask_head][k] is the distance of the k-th selection, in selection
+ *         order; it must be a valid trace: 0 <= o_k <= n_att - 1 + k (0-based k), no repeats.
+ *         mask_heads is 1 (all heads share), H_kv (per kv head) or H_q (per query head, the
+ *         paper's setting; with grouped queries a KV row is read if any head of its group keeps
+ *         it, the other heads ignore it).
+ *   GRID  the trace is generated from the grid instead of being passed: with
+ *         stride = grid_w + row_extra tokens per image row, the column distance of o is
+ *         d(o) = min(o mod stride, stride - o mod stride) and every selection step skips the
+ *         attended key with the largest (d(o), o).  Same mask for all heads.  (Not in the
+ *         paper: a data-free stand-in for its argmin that keeps the diagonals next to the
+ *         multiples of the row stride.)
+ *   WINDOW nothing skipped (n_att is ignored).
+ */
+typedef struct dsa_diag_params {
+    int32_t mode;                 /* dsa_mask_mode                                                 */
+    int32_t window;               /* N_r >= 1                                                      */
+    int32_t n_att;                /* N_att, 1 <= n_att <= window                                   */
+    int32_t grid_w;               /* GRID: image tokens per row                                    */
+    int32_t row_extra;            /* GRID: row-end / separator tokens per row (>= 0)               */
+    const int32_t *skip_offsets;  /* LIST: device [B, mask_heads, trace_len] int32                 */
+    int32_t mask_heads;           /* LIST: 1, H_kv or H_q                                          */
+    int32_t trace_len;            /* LIST: entries per trace, >= window - n_att                    */
+} dsa_diag_params;
+
+/* What a call will launch (filled by dsa_query_plan; for reporting and for tests). */
+typedef struct dsa_plan_info {
+    int32_t split_tokens;   /* kept tokens per thread block                                        */
+    int32_t n_split;        /* splits per (request, kv head); 1 = results written directly         */
+    int32_t launches;       /* kernels launched by the call (1, or 2 with the combine)             */
+    int32_t grid_blocks;    /* thread blocks of the attention kernel                               */
+    int32_t smem_bytes;     /* dynamic shared memory per block                                     */
+    int32_t tile_tokens;    /* tokens per staged K/V tile                                          */
+    int32_t stages;         /* tiles in flight per block                                           */
+} dsa_plan_info;
+
+DSA_API int32_t dsa_version(void);
+DSA_API const char *dsa_status_string(int32_t status);
+/* CUDA error code recorded by the last failing call of this thread (0 if none). */
+DSA_API int32_t dsa_last_cuda_error(void);
+
+/* Bytes of workspace the attention calls need for `problem` (diag == NULL: dense call). */
+DSA_API int32_t dsa_workspace_size(const dsa_problem *problem, const dsa_diag_params *diag, size_t *bytes);
+
+/* The launch plan the attention calls will use for `problem` (diag == NULL: dense call). */
+DSA_API int32_t dsa_query_plan(const dsa_problem *problem, const dsa_diag_params *diag, dsa_plan_info *info);
+
+/*
+ * Dense decode attention (the paper's baseline; Algorithm 1's Attn over every cached token):
+ *   s_j = sm_scale * q_h . k_j  for j in [0, seq_len),  lse = ln sum_j e^{s_j},
+ *   out = sum_j e^{s_j - lse} v_j.
+ * out [B, H_q, D] in problem->dtype; lse [B, H_q] float32, natural log.  A request with
+ * seq_len <= 0 gets out = 0, lse = -inf.
+ */
+DSA_API int32_t dsa_decode_attention_dense(const dsa_problem *problem, void *out, float *lse,
+                                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Diagonal-aware sparse decode attention (Algorithm 1, one step t for every request):
+ *   Attn(Q_t, K_p + K[idx], V_p + V[idx]) with idx = window - skip_idx,
+ * softmax taken jointly over the prompt keys and the kept decode keys.  Only kept rows are read.
+ * Outputs as for the dense call.
+ */
+DSA_API int32_t dsa_decode_attention_sparse(const dsa_problem *problem, const dsa_diag_params *diag,
+                                    void *out, float *lse,
+                                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Merge split-KV partial results (not in the paper; the exact identity that a softmax over a
+ * union of key sets is the lse-weighted mix of the softmaxes over the parts):
+ *   lse = ln sum_i e^{lse_i},  out = sum_i e^{lse_i - lse} out_i.
+ * out_part [B, H_q, n_split, D] float32, lse_part [B, H_q, n_split] float32 (natural log; a
+ * part with lse_i = -inf is empty and its out_i is not read).  out [B, H_q, D] in out_dtype,
+ * lse [B, H_q] float32 (may be NULL).
+ */
+DSA_API int32_t dsa_combine_splits(const float *out_part, const float *lse_part,
+                           int32_t batch, int32_t num_q_heads, int32_t head_dim, int32_t n_split,
+                           void *out, float *lse, int32_t out_dtype, void *stream);
+
+/*
+ * The kept cache positions, produced by the same device code that the sparse attention kernel
+ * uses to decide which rows to read (Algorithm 1: K_p, then window - skip_idx as positions).
+ * idx_out [B, mask_heads, max_kept] int32, ascending, entries beyond the count untouched;
+ * count_out [B, mask_heads] int32 holds the full count even when it exceeds max_kept.
+ * mask_heads is diag->mask_heads for LIST and 1 otherwise; diag == NULL reports the dense set.
+ */
+DSA_API int32_t dsa_debug_kept_indices(const dsa_problem *problem, const dsa_diag_params *diag,
+                               int32_t *idx_out, int32_t *count_out, int32_t max_kept,
+                               void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSA_H */

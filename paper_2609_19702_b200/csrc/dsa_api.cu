@@ -1,0 +1,348 @@
+// C-ABI entry points of the decode-attention library: argument checks, launch planning and
+// kernel dispatch.  Everything here is host code except the kernels it instantiates.
+#include "../../include/dsa.h"
+
+#include <cmath>
+#include <cstdio>
+
+#include "dsa_attn.cuh"
+
+namespace {
+
+using namespace dsa;
+
+thread_local int g_last_cuda_error = 0;
+
+int32_t cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return DSA_ERR_CUDA;
+}
+
+constexpr int kNumSMs = 148;
+constexpr int kMaxDevices = 64;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// The launch plan: how many kept rows one block takes, how many splits that makes.
+struct Plan {
+    int mode;            // MODE_*
+    int G;
+    bool headmask;
+    int tile, stages;
+    int chunk, n_split;
+    int bitmap_words;
+    int64_t grid;
+    size_t smem;
+    size_t ws_out_bytes, ws_total;
+};
+
+template <typename T, int D, int G, bool HM>
+struct KernelPick {
+    static constexpr int TILE = (sizeof(T) == 2 && D == 64) ? 64 : 32;
+    static constexpr int STAGES = (sizeof(T) == 4 && D == 128) ? 3 : 4;
+    using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM>;
+    static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
+    static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
+        auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM>;
+        static bool configured[kMaxDevices] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        }
+        kern<<<(unsigned)grid, NT, smem_bytes, st>>>(a);
+        return cudaGetLastError();
+    }
+};
+
+// Dispatch over (dtype, head_dim, group size, per-head masks).  F(KernelPick<...>) -> R.
+template <class F>
+int32_t dispatch(int dtype, int D, int G, bool hm, F&& f) {
+#define DSA_CASE_G(T, DD)                                                                     \
+    switch (G) {                                                                              \
+        case 1: return f(KernelPick<T, DD, 1, false>{});                                      \
+        case 2: return hm ? f(KernelPick<T, DD, 2, true>{}) : f(KernelPick<T, DD, 2, false>{}); \
+        case 4: return hm ? f(KernelPick<T, DD, 4, true>{}) : f(KernelPick<T, DD, 4, false>{}); \
+        case 8: return hm ? f(KernelPick<T, DD, 8, true>{}) : f(KernelPick<T, DD, 8, false>{}); \
+        default: return DSA_ERR_UNSUPPORTED;                                                  \
+    }
+    if (dtype == DSA_BF16) {
+        if (D == 64) { DSA_CASE_G(__nv_bfloat16, 64) }
+        if (D == 128) { DSA_CASE_G(__nv_bfloat16, 128) }
+    } else if (dtype == DSA_F32) {
+        if (D == 64) { DSA_CASE_G(float, 64) }
+        if (D == 128) { DSA_CASE_G(float, 128) }
+    }
+#undef DSA_CASE_G
+    return DSA_ERR_UNSUPPORTED;
+}
+
+int32_t check_problem(const dsa_problem* p) {
+    if (!p) return DSA_ERR_INVALID_ARG;
+    if (p->batch < 0 || p->num_q_heads < 1 || p->num_kv_heads < 1) return DSA_ERR_INVALID_ARG;
+    if (p->num_q_heads % p->num_kv_heads) return DSA_ERR_INVALID_ARG;
+    if (p->dtype != DSA_BF16 && p->dtype != DSA_F32) return DSA_ERR_UNSUPPORTED;
+    if (p->head_dim != 64 && p->head_dim != 128) return DSA_ERR_UNSUPPORTED;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return DSA_ERR_UNSUPPORTED;
+    if (p->max_seq_len < 0 || p->max_prompt_len < 0 || p->split_tokens < 0) return DSA_ERR_INVALID_ARG;
+    if (!(p->sm_scale >= 0.f) || !std::isfinite(p->sm_scale)) return DSA_ERR_INVALID_ARG;
+    if (p->batch == 0) return DSA_OK;
+    if (!p->q || !p->k_cache || !p->v_cache || !p->seq_len || !p->prompt_len) return DSA_ERR_INVALID_ARG;
+    if (!aligned16(p->q) || !aligned16(p->k_cache) || !aligned16(p->v_cache)) return DSA_ERR_INVALID_ARG;
+    const int64_t vec = p->dtype == DSA_BF16 ? 8 : 4;          // elements per 16 bytes
+    if (p->stride_batch < 0 || p->stride_token < p->head_dim || p->stride_head < 0) return DSA_ERR_INVALID_ARG;
+    if (p->stride_batch % vec || p->stride_token % vec || p->stride_head % vec) return DSA_ERR_INVALID_ARG;
+    if (p->block_table) {
+        if (p->block_size < 1 || p->max_blocks < 1 || p->num_blocks < 1) return DSA_ERR_INVALID_ARG;
+        if ((int64_t)p->max_blocks * p->block_size < p->max_seq_len) return DSA_ERR_INVALID_ARG;
+    }
+    return DSA_OK;
+}
+
+int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
+    if (!d) return DSA_OK;
+    if (d->mode != DSA_MASK_WINDOW && d->mode != DSA_MASK_GRID && d->mode != DSA_MASK_LIST)
+        return DSA_ERR_INVALID_ARG;
+    if (d->window < 1) return DSA_ERR_INVALID_ARG;
+    if (d->mode == DSA_MASK_WINDOW) return DSA_OK;
+    if (d->n_att < 1 || d->n_att > d->window) return DSA_ERR_INVALID_ARG;
+    if (d->mode == DSA_MASK_GRID) {
+        if (d->grid_w < 1 || d->row_extra < 0) return DSA_ERR_INVALID_ARG;
+        if ((int64_t)d->grid_w + d->row_extra > (1 << 30)) return DSA_ERR_INVALID_ARG;
+        return DSA_OK;
+    }
+    if (d->mask_heads != 1 && d->mask_heads != p->num_kv_heads && d->mask_heads != p->num_q_heads)
+        return DSA_ERR_INVALID_ARG;
+    if (d->trace_len < d->window - d->n_att) return DSA_ERR_INVALID_ARG;
+    if (d->window - d->n_att > 0 && p->batch > 0 && !d->skip_offsets) return DSA_ERR_INVALID_ARG;
+    return DSA_OK;
+}
+
+int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
+    int32_t rc = check_problem(p);
+    if (rc != DSA_OK) return rc;
+    rc = check_diag(p, d);
+    if (rc != DSA_OK) return rc;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    pl->G = G;
+    pl->mode = !d ? MODE_DENSE
+                  : (d->mode == DSA_MASK_WINDOW ? MODE_WINDOW : (d->mode == DSA_MASK_GRID ? MODE_GRID : MODE_LIST));
+    // per-query-head masks inside a group: rows of the union are read, heads mask individually
+    pl->headmask = pl->mode == MODE_LIST && G > 1 && d->mask_heads == p->num_q_heads;
+    pl->bitmap_words = pl->mode == MODE_LIST ? (d->window + 31) / 32 : 0;
+
+    // upper bound of kept rows per (request, kv head)
+    int64_t bound = p->max_seq_len;
+    if (d) {
+        const int64_t lp = p->max_prompt_len > 0 ? p->max_prompt_len : p->max_seq_len;
+        int64_t dec = d->window;
+        if (pl->mode != MODE_WINDOW) dec = std::min<int64_t>(d->window, (int64_t)d->n_att * (pl->headmask ? G : 1));
+        bound = std::min<int64_t>(bound, lp + dec);
+    }
+    if (bound < 1) bound = 1;
+
+    size_t smem_probe = 0;
+    rc = dispatch(p->dtype, p->head_dim, G, pl->headmask, [&](auto pick) -> int32_t {
+        using P = decltype(pick);
+        pl->tile = P::TILE;
+        pl->stages = P::STAGES;
+        return DSA_OK;
+    });
+    if (rc != DSA_OK) return rc;
+
+    int chunk;
+    if (p->split_tokens > 0) {
+        chunk = std::min(MAX_CHUNK, round_up(p->split_tokens, pl->tile));
+    } else {
+        // Few (request, kv head) pairs: split until about two waves of blocks exist, but keep
+        // at least a few tiles per block.  Many pairs: as few splits as the row list allows.
+        const int64_t pairs = (int64_t)std::max(p->batch, 1) * p->num_kv_heads;
+        const int64_t target = 2 * 3 * kNumSMs;
+        int64_t want_split = (target + pairs - 1) / pairs;
+        if (want_split < 1) want_split = 1;
+        int64_t c = (bound + want_split - 1) / want_split;
+        c = std::max<int64_t>(c, 4 * pl->tile);
+        chunk = (int)std::min<int64_t>(MAX_CHUNK, round_up((int)std::min<int64_t>(c, MAX_CHUNK), pl->tile));
+    }
+    pl->chunk = chunk;
+    pl->n_split = (int)((bound + chunk - 1) / chunk);
+    pl->grid = (int64_t)p->batch * p->num_kv_heads * pl->n_split;
+    if (pl->grid > 0x7fffffffLL) return DSA_ERR_UNSUPPORTED;
+
+    dispatch(p->dtype, p->head_dim, G, pl->headmask, [&](auto pick) -> int32_t {
+        using P = decltype(pick);
+        smem_probe = P::smem(pl->chunk, pl->bitmap_words);
+        return DSA_OK;
+    });
+    pl->smem = smem_probe;
+    if (pl->smem > 200 * 1024) return DSA_ERR_UNSUPPORTED;     // window too large for LIST bitmaps
+
+    if (pl->n_split > 1) {
+        const size_t rows = (size_t)p->batch * p->num_q_heads * pl->n_split;
+        pl->ws_out_bytes = (rows * p->head_dim * sizeof(float) + 255) / 256 * 256;
+        pl->ws_total = pl->ws_out_bytes + (rows * sizeof(float) + 255) / 256 * 256;
+    } else {
+        pl->ws_out_bytes = 0;
+        pl->ws_total = 0;
+    }
+    return DSA_OK;
+}
+
+void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, AttnArgs* a) {
+    a->q = p->q; a->k = p->k_cache; a->v = p->v_cache;
+    a->stride_b = p->stride_batch; a->stride_tok = p->stride_token; a->stride_head = p->stride_head;
+    a->seq_len = p->seq_len; a->prompt_len = p->prompt_len;
+    a->block_table = p->block_table;
+    a->max_blocks = p->max_blocks; a->block_size = p->block_size; a->num_blocks = p->num_blocks;
+    a->max_seq_len = p->max_seq_len;
+    a->B = p->batch; a->H_q = p->num_q_heads; a->H_kv = p->num_kv_heads;
+    const float scale = p->sm_scale > 0.f ? p->sm_scale : 1.f / sqrtf((float)p->head_dim);
+    a->scale_log2 = scale * LOG2E;
+    a->mask.mode = pl.mode;
+    a->mask.window = d ? d->window : 0;
+    a->mask.n_att = d ? (pl.mode == MODE_WINDOW ? d->window : d->n_att) : 0;
+    a->mask.stride = (d && pl.mode == MODE_GRID) ? d->grid_w + d->row_extra : 1;
+    a->mask.skip_offsets = (d && pl.mode == MODE_LIST) ? d->skip_offsets : nullptr;
+    a->mask.mask_heads = (d && pl.mode == MODE_LIST) ? d->mask_heads : 1;
+    a->mask.trace_len = (d && pl.mode == MODE_LIST) ? d->trace_len : 0;
+    a->mask.bitmap_words = pl.bitmap_words;
+    a->chunk = pl.chunk; a->n_split = pl.n_split;
+    a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
+}
+
+int32_t launch_combine(const float* out_part, const float* lse_part, int64_t rows, int D, int n_split,
+                       void* out, float* lse, int dtype, cudaStream_t st) {
+    if (rows == 0) return DSA_OK;
+    if (dtype == DSA_BF16)
+        dsa_combine_kernel<__nv_bfloat16><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse);
+    else
+        dsa_combine_kernel<float><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+}
+
+int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out, float* lse,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    Plan pl;
+    int32_t rc = make_plan(p, d, &pl);
+    if (rc != DSA_OK) return rc;
+    if (p->batch == 0) return DSA_OK;
+    if (!out || !lse || !aligned16(out)) return DSA_ERR_INVALID_ARG;
+    if (pl.ws_total > 0) {
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return DSA_ERR_INVALID_ARG;
+        if (workspace_bytes < pl.ws_total) return DSA_ERR_WORKSPACE_TOO_SMALL;
+    }
+    AttnArgs a;
+    fill_args(p, d, pl, &a);
+    if (pl.n_split > 1) {
+        a.out_part = reinterpret_cast<float*>(workspace);
+        a.lse_part = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + pl.ws_out_bytes);
+    } else {
+        a.out = out; a.lse = lse;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t err = cudaSuccess;
+    rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, [&](auto pick) -> int32_t {
+        using P = decltype(pick);
+        err = P::launch(a, pl.grid, pl.smem, st);
+        return DSA_OK;
+    });
+    if (rc != DSA_OK) return rc;
+    if (err != cudaSuccess) return cuda_fail(err);
+    if (pl.n_split > 1)
+        return launch_combine(a.out_part, a.lse_part, (int64_t)p->batch * p->num_q_heads, p->head_dim,
+                              pl.n_split, out, lse, p->dtype, st);
+    return DSA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t dsa_version(void) { return DSA_VERSION; }
+
+const char* dsa_status_string(int32_t status) {
+    switch (status) {
+        case DSA_OK: return "ok";
+        case DSA_ERR_INVALID_ARG: return "invalid argument";
+        case DSA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case DSA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case DSA_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
+
+int32_t dsa_workspace_size(const dsa_problem* problem, const dsa_diag_params* diag, size_t* bytes) {
+    if (!bytes) return DSA_ERR_INVALID_ARG;
+    Plan pl;
+    const int32_t rc = make_plan(problem, diag, &pl);
+    if (rc != DSA_OK) return rc;
+    *bytes = pl.ws_total;
+    return DSA_OK;
+}
+
+int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, dsa_plan_info* info) {
+    if (!info) return DSA_ERR_INVALID_ARG;
+    Plan pl;
+    const int32_t rc = make_plan(problem, diag, &pl);
+    if (rc != DSA_OK) return rc;
+    info->split_tokens = pl.chunk;
+    info->n_split = pl.n_split;
+    info->launches = problem->batch == 0 ? 0 : (pl.n_split > 1 ? 2 : 1);
+    info->grid_blocks = (int32_t)pl.grid;
+    info->smem_bytes = (int32_t)pl.smem;
+    info->tile_tokens = pl.tile;
+    info->stages = pl.stages;
+    return DSA_OK;
+}
+
+int32_t dsa_decode_attention_dense(const dsa_problem* problem, void* out, float* lse, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+    return run_attention(problem, nullptr, out, lse, workspace, workspace_bytes, stream);
+}
+
+int32_t dsa_decode_attention_sparse(const dsa_problem* problem, const dsa_diag_params* diag, void* out,
+                                    float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!diag) return DSA_ERR_INVALID_ARG;
+    return run_attention(problem, diag, out, lse, workspace, workspace_bytes, stream);
+}
+
+int32_t dsa_combine_splits(const float* out_part, const float* lse_part, int32_t batch, int32_t num_q_heads,
+                           int32_t head_dim, int32_t n_split, void* out, float* lse, int32_t out_dtype,
+                           void* stream) {
+    if (batch < 0 || num_q_heads < 1 || head_dim < 1 || head_dim > 1024 || n_split < 1) return DSA_ERR_INVALID_ARG;
+    if (out_dtype != DSA_BF16 && out_dtype != DSA_F32) return DSA_ERR_UNSUPPORTED;
+    if (batch == 0) return DSA_OK;
+    if (!out_part || !lse_part || !out) return DSA_ERR_INVALID_ARG;
+    return launch_combine(out_part, lse_part, (int64_t)batch * num_q_heads, head_dim, n_split, out, lse,
+                          out_dtype, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int32_t dsa_debug_kept_indices(const dsa_problem* problem, const dsa_diag_params* diag, int32_t* idx_out,
+                               int32_t* count_out, int32_t max_kept, void* stream) {
+    Plan pl;
+    const int32_t rc = make_plan(problem, diag, &pl);
+    if (rc != DSA_OK) return rc;
+    if (max_kept < 0) return DSA_ERR_INVALID_ARG;
+    if (problem->batch == 0) return DSA_OK;
+    if (!count_out || (max_kept > 0 && !idx_out)) return DSA_ERR_INVALID_ARG;
+    AttnArgs a;
+    fill_args(problem, diag, pl, &a);
+    const int mheads = pl.mode == MODE_LIST ? diag->mask_heads : 1;
+    const size_t smem = (size_t)std::max(pl.bitmap_words, 4) * 4;
+    if (smem > 48 * 1024) return DSA_ERR_UNSUPPORTED;
+    dsa_kept_indices_kernel<<<(unsigned)(problem->batch * mheads), NT, smem,
+                              reinterpret_cast<cudaStream_t>(stream)>>>(a, idx_out, count_out, max_kept);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+}
+
+}  // extern "C"

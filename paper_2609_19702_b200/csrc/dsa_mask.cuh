@@ -1,0 +1,185 @@
+// In-kernel mask generator: turns (decode position, prompt length, window, N_att, grid stride or a
+// skip trace) into the kept cache positions of one request, in ascending order, without touching
+// global memory for anything but the trace.  Used by the attention kernel (to build the list of
+// K/V rows it stages) and by the debug export (to write the positions out).
+//
+// Algorithm 1 of the paper in closed form.  A key chosen for skip_idx at step s with index j has
+// distance o = s - j to the query and keeps it ("+1" shift every step), so with t = p - 1:
+//   window distances  W_t = { 0 .. T },  T = min(t, N_r - 1)
+//   active skips      the first n_act = clamp(t - (N_att - 1), 0, N_r - N_att) selections
+//   kept              prompt [0, L_p)  u  { seq_len - 1 - o : o in W_t \ skips }
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace dsa {
+
+enum : int { MODE_DENSE = 0, MODE_WINDOW = 1, MODE_GRID = 2, MODE_LIST = 3 };
+
+struct MaskArgs {
+    int mode;                  // MODE_*
+    int window;                // N_r
+    int n_att;                 // N_att
+    int stride;                // grid_w + row_extra (GRID)
+    const int* skip_offsets;   // [B, mask_heads, trace_len] (LIST)
+    int mask_heads;
+    int trace_len;
+    int bitmap_words;          // 32-bit words per LIST bitmap = ceil(window / 32)
+};
+
+// Per-request constants of the mask.
+struct ReqMask {
+    int S;        // clamped seq_len
+    int L_p;      // clamped prompt length
+    int p;        // decode tokens in the cache, current one included
+    int T;        // largest window distance
+    int n_win;    // window candidates = T + 1 (0 when p == 0)
+    int w_lo;     // cache position of distance T
+    int n_act;    // LIST: active skip entries
+    int dstar;    // GRID: column distance of the partly kept class (-1: keep none below T)
+    int need;     // GRID: how many distances of class dstar are kept (lowest first)
+    bool keep_all;// nothing skipped at this position
+};
+
+// Number of distances o in [0, T) whose column distance is <= x.
+__device__ __forceinline__ int grid_count_le(int T, int stride, int x) {
+    if (2 * x + 1 >= stride) return T;
+    const int full = T / stride, rem = T - full * stride;
+    const int hi_start = stride - x;                     // r >= stride - x  (and r > x here)
+    const int part = min(rem, x + 1) + max(0, rem - hi_start);
+    return full * (2 * x + 1) + part;
+}
+
+__device__ __forceinline__ ReqMask req_mask_setup(const MaskArgs& a, int seq_len, int prompt_len,
+                                                  int max_seq_len) {
+    ReqMask m;
+    m.S = max(0, min(seq_len, max_seq_len));
+    m.L_p = max(0, min(prompt_len, m.S));
+    m.p = m.S - m.L_p;
+    m.n_act = 0; m.dstar = -1; m.need = 0; m.keep_all = true;
+    if (a.mode == MODE_DENSE) {
+        m.T = m.p - 1; m.n_win = m.p; m.w_lo = m.L_p;
+        return m;
+    }
+    const int t = m.p - 1;
+    m.T = min(t, a.window - 1);
+    m.n_win = m.p > 0 ? m.T + 1 : 0;
+    m.w_lo = m.S - m.n_win;
+    if (a.mode == MODE_WINDOW || m.p == 0 || t < a.n_att - 1) return m;   // phase 1 / nothing to skip
+    if (a.mode == MODE_LIST) {
+        m.n_act = min(min(t - (a.n_att - 1), a.window - a.n_att), a.trace_len);
+        m.keep_all = m.n_act <= 0;
+        return m;
+    }
+    // GRID: keep the N_att - 1 best of [0, T) under (column distance, distance), plus T itself.
+    m.keep_all = false;
+    const int want = a.n_att - 1;
+    if (want <= 0) { m.dstar = -1; m.need = 0; return m; }
+    int lo = 0, hi = a.stride / 2;                       // smallest x with count_le(x) >= want
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (grid_count_le(m.T, a.stride, mid) >= want) hi = mid; else lo = mid + 1;
+    }
+    m.dstar = lo;
+    m.need = want - (lo > 0 ? grid_count_le(m.T, a.stride, lo - 1) : 0);
+    return m;
+}
+
+__device__ __forceinline__ bool grid_keep(const ReqMask& m, int stride, int o) {
+    if (o == m.T) return true;
+    const int k = o / stride, r = o - k * stride;
+    const int d = min(r, stride - r);
+    if (d != m.dstar) return d < m.dstar;
+    const int rank = (m.dstar == 0 || 2 * m.dstar == stride) ? k : 2 * k + (r == m.dstar ? 0 : 1);
+    return rank < m.need;
+}
+
+// LIST: set the bits of the active skip distances of one trace in a shared-memory bitmap
+// (cleared by the caller).  Distances outside [0, window) are ignored.
+template <int NT>
+__device__ __forceinline__ void list_bitmap_fill(const MaskArgs& a, const ReqMask& m,
+                                                 const int* trace, unsigned* bitmap) {
+    for (int i = threadIdx.x; i < m.n_act; i += NT) {
+        const int o = trace[i];
+        if (o >= 0 && o < a.window) atomicOr(&bitmap[o >> 5], 1u << (o & 31));
+    }
+}
+
+// Which of the `slots` masks (one per head that shares this KV row) keep distance o.
+template <int SLOTS>
+__device__ __forceinline__ unsigned keep_bits(const MaskArgs& a, const ReqMask& m,
+                                              const unsigned* bitmaps, int o) {
+    constexpr unsigned ALL = (1u << SLOTS) - 1u;
+    if (m.keep_all) return ALL;
+    if (a.mode == MODE_GRID) return grid_keep(m, a.stride, o) ? ALL : 0u;
+    unsigned bits = 0;
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+        const unsigned w = bitmaps[s * a.bitmap_words + (o >> 5)];
+        bits |= (((w >> (o & 31)) & 1u) ^ 1u) << s;
+    }
+    return bits;
+}
+
+// Exclusive scan of one int per thread over a block of NT threads (NT a multiple of 32).
+template <int NT>
+__device__ __forceinline__ int block_excl_scan(int v, int& total, int* s_warp /* [NT/32] */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += n;
+    }
+    __syncthreads();                      // s_warp may still be read from a previous use
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) {
+        const int c = s_warp[w];
+        if (w < warp) base += c;
+        tot += c;
+    }
+    total = tot;
+    return base + incl - v;
+}
+
+// Enumerate the kept positions with union rank in [r0, r1), calling
+//   sink(rank - r0, cache position, head bits)
+// for each, and return the total number of kept positions (union over the SLOTS masks).
+// All NT threads of the block must call it (it synchronises).
+template <int NT, int SLOTS, class Sink>
+__device__ __forceinline__ int enumerate_kept(const MaskArgs& a, const ReqMask& m,
+                                              const unsigned* bitmaps, int r0, int r1,
+                                              int* s_warp, Sink sink) {
+    constexpr unsigned ALL = (1u << SLOTS) - 1u;
+    // the prompt: always attended in full
+    for (int r = max(r0, 0) + (int)threadIdx.x; r < min(r1, m.L_p); r += NT) sink(r - r0, r, ALL);
+    if (m.keep_all) {
+        // contiguous window: rank L_p + c  <->  position w_lo + c
+        const int lo = max(r0, m.L_p), hi = min(r1, m.L_p + m.n_win);
+        for (int r = lo + (int)threadIdx.x; r < hi; r += NT) sink(r - r0, m.w_lo + (r - m.L_p), ALL);
+        return m.L_p + m.n_win;
+    }
+    // Each thread owns a contiguous run of window candidates (ascending position = descending
+    // distance): count, scan, then emit.
+    const int per = (m.n_win + NT - 1) / NT;
+    const int c0 = min((int)threadIdx.x * per, m.n_win), c1 = min(c0 + per, m.n_win);
+    int cnt = 0;
+    for (int c = c0; c < c1; ++c) cnt += keep_bits<SLOTS>(a, m, bitmaps, m.T - c) != 0u;
+    int total;
+    int rank = m.L_p + block_excl_scan<NT>(cnt, total, s_warp);
+    if (rank < r1 && rank + cnt > r0) {
+        for (int c = c0; c < c1; ++c) {
+            const unsigned bits = keep_bits<SLOTS>(a, m, bitmaps, m.T - c);
+            if (bits) {
+                if (rank >= r0 && rank < r1) sink(rank - r0, m.w_lo + c, bits);
+                ++rank;
+            }
+        }
+    }
+    return m.L_p + total;
+}
+
+}  // namespace dsa

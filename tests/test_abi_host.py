@@ -1,0 +1,116 @@
+"""Host-only checks of the C-ABI library: it loads, exports every symbol the header declares,
+and rejects bad arguments before touching a device.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "dsa.h")
+
+
+@pytest.fixture(scope="module")
+def dsa():
+    from paper_2609_19702_b200 import build
+    build.build()
+    from paper_2609_19702_b200 import binding
+    return binding
+
+
+def _declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dsa_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(dsa):
+    names = _declared_functions()
+    assert "dsa_decode_attention_dense" in names and "dsa_decode_attention_sparse" in names
+    assert "dsa_combine_splits" in names
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), "libdsa.so does not export %s" % n
+    assert sorted(names) == sorted(dsa.EXPORTS)
+    for n in names:
+        assert hasattr(dsa, n) or n in ("dsa_status_string", "dsa_last_cuda_error"), n
+
+
+def test_version_and_status_strings(dsa):
+    assert dsa.dsa_version() == 100
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    lib.dsa_status_string.restype = ctypes.c_char_p
+    assert lib.dsa_status_string(0) == b"ok"
+    assert lib.dsa_status_string(-3) == b"workspace too small"
+
+
+def _problem(dsa, **kw):
+    p = dsa.dsa_problem()
+    p.batch, p.num_q_heads, p.num_kv_heads, p.head_dim = 4, 32, 8, 128
+    p.dtype = dsa.DSA_BF16
+    # fake, aligned, never dereferenced on the host
+    p.q = p.k_cache = p.v_cache = 0x10000
+    p.seq_len = p.prompt_len = 0x20000
+    p.stride_batch, p.stride_token, p.stride_head = 8254 * 1024, 1024, 128
+    p.max_seq_len, p.max_prompt_len = 8254, 64
+    for k, v in kw.items():
+        setattr(p, k, v)
+    return p
+
+
+def _plan(dsa, p, d=None):
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    info = dsa.dsa_plan_info()
+    rc = lib.dsa_query_plan(ctypes.byref(p), ctypes.byref(d) if d is not None else None, ctypes.byref(info))
+    return rc, info
+
+
+def _diag(dsa, **kw):
+    d = dsa.dsa_diag_params()
+    d.mode, d.window, d.n_att, d.grid_w, d.row_extra = dsa.DSA_MASK_GRID, 1024, 410, 90, 1
+    for k, v in kw.items():
+        setattr(d, k, v)
+    return d
+
+
+def test_argument_validation_on_host(dsa):
+    ok, info = _plan(dsa, _problem(dsa))
+    assert ok == 0 and info.n_split >= 1 and info.split_tokens % info.tile_tokens == 0
+    assert _plan(dsa, _problem(dsa, head_dim=96))[0] == -2
+    assert _plan(dsa, _problem(dsa, num_kv_heads=5))[0] == -1
+    assert _plan(dsa, _problem(dsa, num_q_heads=48, num_kv_heads=16))[0] == -2      # group of 3
+    assert _plan(dsa, _problem(dsa, q=0))[0] == -1
+    assert _plan(dsa, _problem(dsa, k_cache=0x10004))[0] == -1                    # misaligned
+    assert _plan(dsa, _problem(dsa, stride_token=100))[0] == -1
+    assert _plan(dsa, _problem(dsa, stride_head=12))[0] == -1
+    assert _plan(dsa, _problem(dsa, dtype=7))[0] == -2
+    assert _plan(dsa, _problem(dsa, block_table=0x30000, block_size=16, max_blocks=10, num_blocks=99))[0] == -1
+    assert _plan(dsa, _problem(dsa), _diag(dsa, n_att=2000))[0] == -1
+    assert _plan(dsa, _problem(dsa), _diag(dsa, window=0))[0] == -1
+    assert _plan(dsa, _problem(dsa), _diag(dsa, grid_w=0))[0] == -1
+    assert _plan(dsa, _problem(dsa), _diag(dsa, mode=dsa.DSA_MASK_LIST, mask_heads=3, trace_len=614,
+                                           skip_offsets=0x40000))[0] == -1
+    assert _plan(dsa, _problem(dsa), _diag(dsa, mode=dsa.DSA_MASK_LIST, mask_heads=32, trace_len=10,
+                                           skip_offsets=0x40000))[0] == -1
+
+
+def test_plan_sizes(dsa):
+    # sparse: prompt + N_att rows per kv head fit one block -> no split, one launch
+    rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,
+                                   max_prompt_len=200), _diag(dsa, window=512, n_att=208, grid_w=64))
+    assert rc == 0 and info.n_split == 1 and info.launches == 1 and info.grid_blocks == 256 * 32
+    # dense on the same problem needs splits and the combine kernel
+    rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360))
+    assert rc == 0 and info.n_split * info.split_tokens >= 4360 and info.launches == 2
+    # workspace covers the partials
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    n = ctypes.c_size_t(0)
+    p = _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360)
+    assert lib.dsa_workspace_size(ctypes.byref(p), None, ctypes.byref(n)) == 0
+    assert n.value >= 256 * 32 * info.n_split * (128 + 1) * 4
+    # explicit split size is honoured, rounded to the tile
+    rc, info = _plan(dsa, _problem(dsa, split_tokens=100))
+    assert rc == 0 and info.split_tokens == 128
+    # a few requests with long sequences are split to fill the machine
+    rc, info = _plan(dsa, _problem(dsa, batch=1))
+    assert rc == 0 and info.grid_blocks >= 148
