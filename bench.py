@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-attention hot path.
+
+    python bench.py --gpus 1 --steps K --warmup W            # this library (CUDA, sm_100a)
+    python bench.py --impl reference --steps K --warmup W    # the float64 CPU oracle
+
+A "step" is one sparse decode-attention call (mask generation, K/V staging, scores, online
+softmax, partial write and split combine where the plan needs one) over one batch of the paged
+throughput workload at its largest batch: 256 requests, 32/32 heads, head_dim 128, bf16, 200
+prompt tokens + a 64x64 grid with one separator per row, 16-token blocks in a shuffled block
+table, decode positions uniform in [1, 4160], window 512 / N_att 208.  Inputs are seeded and
+synthetic and already resident in HBM when the timed region starts; every step reads ~1.7 GB of
+distinct K/V, far more than the L2, so no flush is needed between steps.
+
+One JSON line is printed by rank 0.  With torchrun (N > 1) every rank owns its own batch of the
+same shape (requests are independent: weak scaling, no collective on the data path) and the
+time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "decode_attention_queries_per_sec"
+UNIT = "queries/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per launch of the timed kernel from an ncu capture (see profiles/), keyed by the
+# workload string of the JSON line; None until a capture of that exact launch exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=5, help="workload 1..5")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--window", type=int, default=None)
+    ap.add_argument("--n-att", type=int, default=None)
+    ap.add_argument("--mode", default="sparse", choices=["sparse", "dense"])
+    ap.add_argument("--split-tokens", type=int, default=0)
+    ap.add_argument("--no-variants", action="store_true", help="skip the dense / other-window timings")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def workload_name(w, mode):
+    s = "config%d_%s B=%d Hq=%d Hkv=%d D=%d Lp=%d grid=%dx%d+%d %s" % (
+        w.index, w.name, w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.prompt_len,
+        w.grid_h, w.grid_w, w.row_extra, "paged%d" % w.block_size if w.paged else "contiguous")
+    if mode == "sparse":
+        s += " sparse grid-mask window=%d n_att=%d" % (w.window, w.n_att)
+    else:
+        s += " dense"
+    return s
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, torch_device_index: int):
+        self.samples, self.reasons, self.max_mhz, self.err = [], set(), None, None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            props = torch.cuda.get_device_properties(torch_device_index)
+            handle = None
+            try:
+                bus = "%08x:%02x:%02x.0" % (props.pci_domain_id, props.pci_bus_id, props.pci_device_id)
+                handle = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = torch_device_index
+                if vis:
+                    try:
+                        idx = int(vis.split(",")[torch_device_index])
+                    except ValueError:
+                        pass
+                handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self._nv, self._h = pynvml, handle
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # pragma: no cover
+            self.err = repr(e)
+            self._nv = None
+
+    def _run(self):
+        nv, h = self._nv, self._h
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception as e:  # pragma: no cover
+                self.err = repr(e)
+                break
+            time.sleep(0.002)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        out = {"sm_mhz": int(np.median(self.samples)) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if self.err:
+            out["error"] = self.err
+        return out
+
+
+def algorithmic_bytes(w, host, mode, blocks_touched):
+    """Bytes one call must move: kept K and V rows, q, out, lse, and the block-table entries of
+    the blocks it touches.  Kept rows per kv head: the whole prompt plus min(p, N_att) decode
+    keys for the sparse call (the attended count of Algorithm 1), p for the dense call."""
+    esize = 2
+    p = host["position"].astype(np.int64)
+    lp = host["prompt_len"].astype(np.int64)
+    dec = p if mode == "dense" else np.minimum(p, w.n_att)
+    kept_rows = int((lp + dec).sum())
+    kv = kept_rows * w.num_kv_heads * w.head_dim * esize * 2
+    qo = w.batch * w.num_q_heads * (2 * w.head_dim * esize + 4)
+    table = 4 * int(blocks_touched)
+    return kv + qo + table, kept_rows
+
+
+def time_calls(torch, fn, steps, warmup, sampler=None, barrier=None):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+        torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    return e0.elapsed_time(e1) / 1e3, clocks          # seconds for `steps` calls
+
+
+def run_ours(args):
+    import torch
+    from paper_2609_19702_b200 import build as cuda_build
+    cuda_build.build()
+    from paper_2609_19702_b200 import binding as dsa, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    w = synth.workload(args.config, batch=args.batch, window=args.window, n_att=args.n_att)
+    inputs = synth.make_inputs_device(w, dev, seed=synth.BASE_SEED + w.index + 1000 * rank)
+    host = inputs["host"]
+
+    def problem(split_tokens=0):
+        return dsa.Problem(
+            q=inputs["q"], k_cache=inputs["k_cache"], v_cache=inputs["v_cache"], strides=inputs["strides"],
+            seq_len=inputs["seq_len"], prompt_len=inputs["prompt_len"], num_kv_heads=w.num_kv_heads,
+            max_seq_len=inputs["max_seq_len"], max_prompt_len=w.prompt_len,
+            block_table=inputs["block_table"], block_size=inputs["block_size"],
+            num_blocks=0 if inputs["block_table"] is None else inputs["block_table"].numel(),
+            split_tokens=split_tokens)
+
+    prob = problem(args.split_tokens)
+    out, lse = dsa.alloc_outputs(prob)
+
+    def make_call(mode, ww):
+        diag = None if mode == "dense" else dsa.Diag(dsa.DSA_MASK_GRID, ww.window, ww.n_att, ww.grid_w, ww.row_extra)
+        ws = dsa.alloc_workspace(prob, diag)
+        plan = dsa.dsa_query_plan(prob, diag)
+        if diag is None:
+            return (lambda: dsa.dsa_decode_attention_dense(prob, out, lse, ws)), plan, diag
+        return (lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)), plan, diag
+
+    # ---- the timed step ------------------------------------------------------------------
+    call, plan, diag = make_call(args.mode, w)
+    sampler = ClockSampler(local_rank)
+    secs, clocks = time_calls(torch, call, args.steps, args.warmup, sampler, barrier)
+    t = torch.tensor([secs], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    secs_max = float(t.item())
+    ms_per_step = secs_max / args.steps * 1e3
+    value = world * w.batch * args.steps / secs_max
+
+    # ---- roofline of the attention kernel (rank-local numbers) ----------------------------
+    idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, inputs["max_seq_len"])
+    torch.cuda.synchronize()
+    if inputs["block_table"] is not None:
+        valid = torch.arange(idx.shape[2], device=dev)[None, None, :] < cnt[:, :, None]
+        blk = torch.where(valid, idx // inputs["block_size"], -1)
+        blocks_touched = sum(int(torch.unique(blk[i][blk[i] >= 0]).numel()) for i in range(blk.shape[0]))
+    else:
+        blocks_touched = 0
+    del idx
+    abytes, kept_rows = algorithmic_bytes(w, host, args.mode, blocks_touched)
+    peak, peak_kind = measured_peak()
+    launch_secs = secs / args.steps                       # one attention launch (+ combine) per step
+    achieved = abytes / launch_secs / 1e9
+    name = workload_name(w, args.mode)
+    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(name),
+                "peak_kind": "of " + peak_kind, "algorithmic_bytes": abytes,
+                "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+                "kernel": "dsa_attn_kernel" + (" + dsa_combine_kernel" if plan.launches > 1 else "")}
+
+    # ---- variants: dense and the other window, same library, same batch --------------------
+    variants = {}
+    if not args.no_variants and args.mode == "sparse":
+        vsteps = max(5, args.steps // 10)
+        todo = [("dense", w)]
+        if w.index == 5:
+            todo.append(("sparse", synth.workload(5, batch=w.batch, window=1024, n_att=416)))
+        for mode, ww in todo:
+            vcall, vplan, _ = make_call(mode, ww)
+            vsecs, _ = time_calls(torch, vcall, vsteps, 3)
+            vb, _ = algorithmic_bytes(ww, host, mode, 0)
+            key = "dense" if mode == "dense" else "sparse_w%d_a%d" % (ww.window, ww.n_att)
+            variants[key] = {"ms_per_step": round(vsecs / vsteps * 1e3, 4),
+                             "queries_per_sec": round(w.batch * vsteps / vsecs, 1),
+                             "achieved_GBs": round(vb / (vsecs / vsteps) / 1e9, 1),
+                             "frac_of_peak": round(vb / (vsecs / vsteps) / 1e9 / peak, 4),
+                             "launches_per_step": vplan.launches, "n_split": vplan.n_split}
+        if "dense" in variants:
+            variants["sparse_over_dense_speedup"] = round(variants["dense"]["ms_per_step"] / (launch_secs * 1e3), 3)
+            dense_bytes, _ = algorithmic_bytes(w, host, "dense", 0)
+            variants["ideal_byte_ratio"] = round(dense_bytes / abytes, 3)
+
+    # ---- end to end: per-step inputs from pinned host memory, result back to the host ------
+    e2e = None
+    if not args.no_e2e:
+        h_q = inputs["q"].cpu().pin_memory()
+        h_seq = inputs["seq_len"].cpu().pin_memory()
+        h_pl = inputs["prompt_len"].cpu().pin_memory()
+        h_bt = None if inputs["block_table"] is None else inputs["block_table"].cpu().pin_memory()
+        h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        h_lse = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+
+        def e2e_step():
+            inputs["q"].copy_(h_q, non_blocking=True)
+            inputs["seq_len"].copy_(h_seq, non_blocking=True)
+            inputs["prompt_len"].copy_(h_pl, non_blocking=True)
+            if h_bt is not None:
+                inputs["block_table"].copy_(h_bt, non_blocking=True)
+            call()
+            h_out.copy_(out, non_blocking=True)
+            h_lse.copy_(lse, non_blocking=True)
+            torch.cuda.current_stream().synchronize()      # the caller needs the result to go on
+
+        esteps = min(args.steps, 100)
+        esecs, _ = time_calls(torch, e2e_step, esteps, 3, None, barrier)
+        te = torch.tensor([esecs], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        h2d = sum(x.numel() * x.element_size() for x in (h_q, h_seq, h_pl) + ((h_bt,) if h_bt is not None else ()))
+        d2h = h_out.numel() * h_out.element_size() + h_lse.numel() * h_lse.element_size()
+        e2e = {"value": round(world * w.batch * esteps / float(te.item()), 1), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": esteps,
+               "note": "per step: q, seq_len, prompt_len and block table from pinned host memory, "
+                       "out and lse back to pinned host memory, stream synchronised; the KV cache is "
+                       "decode state and stays resident in HBM"}
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload ------------------
+    cpu = None
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        cpu = oracle_baseline(synth, inputs, w, args.mode)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": name, "global_batch": world * w.batch,
+                       "kept_rows_per_kv_head_mean": round(kept_rows / w.batch, 1),
+                       "l2": "inputs larger than L2: each step reads %.2f GB of distinct K/V" % (abytes / 1e9),
+                       "parallelism": "requests sharded over %d GPU(s), no collective" % world,
+                       "plan": {"split_tokens": plan.split_tokens, "n_split": plan.n_split,
+                                "grid_blocks": plan.grid_blocks, "smem_bytes": plan.smem_bytes,
+                                "tile_tokens": plan.tile_tokens, "stages": plan.stages}},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def oracle_baseline(synth, inputs, w, mode, sample=16, min_seconds=10.0):
+    """Time the float64 oracle, as it stands, on the first `sample` requests of this batch."""
+    from oracle import oracle as ora
+    n = min(sample, w.batch)
+    sub = synth.host_subset(inputs, range(n))
+    kw = dict(num_kv_heads=w.num_kv_heads, strides=sub["strides"], block_table=sub["block_table"],
+              block_size=sub["block_size"])
+    if mode == "dense":
+        kw.update(mode=ora.MODE_DENSE)
+    else:
+        kw.update(mode=ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride_grid=w.stride)
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        ora.decode(sub["q"], sub["k_cache"], sub["v_cache"], sub["seq_len"], sub["prompt_len"], **kw)
+        reps += 1
+        el = time.perf_counter() - t0
+        if el >= min_seconds or reps >= 1000:
+            break
+    return {"value": round(n * reps / el, 2), "unit": UNIT, "cores": ora.num_threads(), "kind": "oracle",
+            "sample": "first %d requests of the batch, %d repetitions, %.1f s" % (n, reps, el)}
+
+
+def run_reference(args):
+    """The reference arm: the float64 CPU oracle on the same workload, metric and unit; each step
+    is one oracle call on a bounded sample of requests.  Rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import oracle as ora
+    from paper_2609_19702_b200 import synth
+    sample = 4
+    w_full = synth.workload(args.config, batch=args.batch, window=args.window, n_att=args.n_att)
+    w = synth.workload(args.config, batch=sample, window=args.window, n_att=args.n_att)
+    inp = synth.make_inputs(w)
+    kw = dict(num_kv_heads=w.num_kv_heads, strides=inp["strides"], block_table=inp["block_table"],
+              block_size=inp["block_size"])
+    if args.mode == "dense":
+        kw.update(mode=ora.MODE_DENSE)
+    else:
+        kw.update(mode=ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride_grid=w.stride)
+
+    def step():
+        ora.decode(inp["q"], inp["k_cache"], inp["v_cache"], inp["seq_len"], inp["prompt_len"], **kw)
+
+    steps = min(args.steps, 50)
+    for _ in range(min(args.warmup, 3)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    el = time.perf_counter() - t0
+    value = round(sample * steps / el, 2)
+    cpu = {"value": value, "unit": UNIT, "cores": ora.num_threads(), "kind": "oracle",
+           "sample": "%d requests of the workload per step, %d steps" % (sample, steps)}
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 3), "ms_per_step": round(el / steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": workload_name(w_full, args.mode)},
+        "cpu_baseline": cpu,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -212,3 +212,133 @@ def shard_requests(batch: int, world_size: int, rank: int) -> range:
     base, extra = divmod(batch, world_size)
     lo = rank * base + min(rank, extra)
     return range(lo, lo + base + (1 if rank < extra else 0))
+
+
+def make_inputs_device(w: Workload, device, seed: Optional[int] = None) -> Dict[str, object]:
+    """Full-size batches for benchmarking: same shapes, layouts and position mix as
+    ``make_inputs`` but K/V/q are drawn on ``device`` with a seeded torch generator (a paged pool
+    at batch 256 is 18 GB, too slow to draw on the host).  Values are N(0,1) (+ the positional
+    component where the workload has one) rounded to bf16.  Returns torch tensors; positions,
+    lengths and the block table are also returned as numpy arrays under ``host``.
+    """
+    import torch
+
+    seed = BASE_SEED + w.index if seed is None else seed
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    b, hq, hkv, d = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    s_max = w.max_seq_len
+    row = hkv * d
+    if w.share_cache:
+        position = (np.arange(b, dtype=np.int32) % w.image_tokens) + 1
+    else:
+        position = rng.integers(w.pos_lo, w.pos_hi + 1, size=b, dtype=np.int32)
+    prompt_len = np.full(b, w.prompt_len, dtype=np.int32)
+    seq_len = (prompt_len + position).astype(np.int32)
+    pos_emb = torch.from_numpy(_positional(w)).to(device) if w.positional else None
+
+    q = torch.randn((b, hq, d), generator=gen, device=device, dtype=torch.float32)
+    if pos_emb is not None:
+        q += pos_emb[torch.from_numpy(position.astype(np.int64) - 1).to(device)][:, None, :]
+    q = q.to(torch.bfloat16)
+
+    def draw(n_seq: int):
+        """[n_seq, s_pad, hkv, d] bf16, one sequence at a time to bound temporaries."""
+        s_pad = s_max if not w.paged else ((s_max + w.block_size - 1) // w.block_size) * w.block_size
+        out = torch.empty((n_seq, s_pad, hkv, d), device=device, dtype=torch.bfloat16)
+        for i in range(n_seq):
+            x = torch.randn((s_pad, hkv, d), generator=gen, device=device, dtype=torch.float32)
+            if pos_emb is not None:
+                x[w.prompt_len:s_max] += pos_emb[:, None, :]
+            out[i] = x.to(torch.bfloat16)
+        return out
+
+    block_table = None
+    if w.paged:
+        bs = w.block_size
+        max_blocks = (s_max + bs - 1) // bs
+        num_blocks = b * max_blocks
+        block_table = rng.permutation(num_blocks).astype(np.int32).reshape(b, max_blocks)
+        if not w.positional:
+            # the pool is i.i.d. noise, so drawing it in pool order is the same distribution as
+            # drawing per sequence and scattering through the table
+            k_cache = draw(b).reshape(num_blocks, bs, hkv, d)
+            v_cache = draw(b).reshape(num_blocks, bs, hkv, d)
+        else:
+            bt = torch.from_numpy(block_table.astype(np.int64)).to(device)
+            k_cache = torch.empty((num_blocks, bs, hkv, d), device=device, dtype=torch.bfloat16)
+            v_cache = torch.empty_like(k_cache)
+            for i in range(b):
+                k_cache[bt[i]] = draw(1).reshape(max_blocks, bs, hkv, d)
+                v_cache[bt[i]] = draw(1).reshape(max_blocks, bs, hkv, d)
+        strides = (bs * row, row, d)
+    elif w.share_cache:
+        k_cache, v_cache = draw(1), draw(1)
+        strides = (0, row, d)
+    else:
+        k_cache, v_cache = draw(b), draw(b)
+        strides = (s_max * row, row, d)
+
+    return {
+        "workload": w,
+        "q": q,
+        "k_cache": k_cache.reshape(-1),
+        "v_cache": v_cache.reshape(-1),
+        "cache_shape": tuple(k_cache.shape),
+        "strides": strides,
+        "seq_len": torch.from_numpy(seq_len).to(device),
+        "prompt_len": torch.from_numpy(prompt_len).to(device),
+        "block_table": None if block_table is None else torch.from_numpy(block_table).to(device),
+        "block_size": w.block_size if w.paged else 0,
+        "max_seq_len": s_max,
+        "host": {"seq_len": seq_len, "prompt_len": prompt_len, "position": position.astype(np.int32),
+                 "block_table": block_table},
+    }
+
+
+def host_subset(dev: Dict[str, object], requests) -> Dict[str, object]:
+    """Copy the given requests of a device batch (``make_inputs_device``) to the host, in the
+    dict layout of ``make_inputs`` (bf16 bit patterns; paged pools are compacted to the blocks
+    these requests own and the block table renumbered).  Pure data movement."""
+    import torch
+
+    w: Workload = dev["workload"]
+    req = [int(r) for r in requests]
+    n = len(req)
+    hkv, d = w.num_kv_heads, w.head_dim
+    ridx = torch.tensor(req, dtype=torch.int64, device=dev["q"].device)
+
+    def bits(t):
+        return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+    host = dev["host"]
+    out = {
+        "workload": replace(w, batch=n, share_cache=False) if not w.share_cache else replace(w, batch=n),
+        "q": bits(dev["q"][ridx]),
+        "seq_len": host["seq_len"][req].copy(),
+        "prompt_len": host["prompt_len"][req].copy(),
+        "position": host["position"][req].copy(),
+        "block_size": dev["block_size"],
+        "max_seq_len": dev["max_seq_len"],
+        "block_table": None,
+    }
+    if w.paged:
+        bs = w.block_size
+        bt = dev["block_table"][ridx].to(torch.int64)
+        max_blocks = bt.shape[1]
+        kc = dev["k_cache"].view(-1, bs, hkv, d)[bt.reshape(-1)]
+        vc = dev["v_cache"].view(-1, bs, hkv, d)[bt.reshape(-1)]
+        out["k_cache"], out["v_cache"] = bits(kc).reshape(-1), bits(vc).reshape(-1)
+        out["block_table"] = np.arange(n * max_blocks, dtype=np.int32).reshape(n, max_blocks)
+        out["strides"] = dev["strides"]
+    elif w.share_cache:
+        out["k_cache"], out["v_cache"] = bits(dev["k_cache"]).reshape(-1), bits(dev["v_cache"]).reshape(-1)
+        out["strides"] = dev["strides"]
+    else:
+        s_max = dev["max_seq_len"]
+        kc = dev["k_cache"].view(-1, s_max, hkv, d)[ridx]
+        vc = dev["v_cache"].view(-1, s_max, hkv, d)[ridx]
+        out["k_cache"], out["v_cache"] = bits(kc).reshape(-1), bits(vc).reshape(-1)
+        out["strides"] = dev["strides"]
+    return out
