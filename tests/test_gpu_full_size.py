@@ -1,0 +1,56 @@
+"""Parity at the benchmark's full size and launch configuration: the paged throughput workload
+at batch 256 (18 GB of K/V drawn on the device), checked on sampled requests that the oracle
+computes one by one from a host copy of just their blocks."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as ora
+from paper_2609_19702_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config5_batch256_sampled_requests():
+    from paper_2609_19702_b200 import binding as dsa
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24 << 30:
+        pytest.skip("needs 24 GB of free device memory")
+    w = synth.workload(5, batch=256)
+    dev = synth.make_inputs_device(w, torch.device("cuda"))
+    prob = dsa.Problem(q=dev["q"], k_cache=dev["k_cache"], v_cache=dev["v_cache"], strides=dev["strides"],
+                       seq_len=dev["seq_len"], prompt_len=dev["prompt_len"], num_kv_heads=w.num_kv_heads,
+                       max_seq_len=dev["max_seq_len"], max_prompt_len=w.prompt_len,
+                       block_table=dev["block_table"], block_size=dev["block_size"],
+                       num_blocks=dev["block_table"].numel())
+    pos = dev["host"]["position"]
+    # shortest, longest, around the phase boundaries of both windows, and a few at random
+    order = np.argsort(pos)
+    sample = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]),
+                     int(np.argmin(np.abs(pos - 208))), int(np.argmin(np.abs(pos - 512))),
+                     int(np.argmin(np.abs(pos - 1024))), 0, 17, 101, 255})
+    sub = synth.host_subset(dev, sample)
+    out, lse = dsa.alloc_outputs(prob)
+    sidx = torch.tensor(sample, device="cuda")
+
+    cases = [(None, ora.MODE_DENSE, dict())]
+    for window, n_att in ((512, 208), (1024, 416)):
+        cases.append((dsa.Diag(dsa.DSA_MASK_GRID, window, n_att, w.grid_w, w.row_extra), ora.MODE_GRID,
+                      dict(n_r=window, n_att=n_att, stride=w.stride)))
+    for diag, mode, kw in cases:
+        out.fill_(float("nan"))
+        ws = dsa.alloc_workspace(prob, diag)
+        if diag is None:
+            dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+        else:
+            dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+        torch.cuda.synchronize()
+        assert torch.isfinite(out.float()).all()
+        ref = util.oracle_run(sub, mode, want_kept=True, **kw)
+        util.assert_close(out[sidx], lse[sidx], ref, what="full size mode %d" % mode)
+        idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, dev["max_seq_len"])
+        util.assert_kept_equal(idx[sidx], cnt[sidx], ref, "full size mode %d" % mode)
+        # property that holds for every request: kept count = prompt + min(p, N_att) (or p)
+        want = w.prompt_len + (pos if diag is None else np.minimum(pos, diag.n_att))
+        assert np.array_equal(cnt.cpu().numpy()[:, 0], want)
