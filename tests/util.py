@@ -41,7 +41,8 @@ def assert_close(out_gpu, lse_gpu, ref, f32=False, what=""):
         what, err.max(), np.unravel_index(err.argmax(), err.shape))
     ref_lse = ref["lse"]
     both_inf = np.isneginf(lse) & np.isneginf(ref_lse)
-    lerr = np.where(both_inf, 0.0, np.abs(lse - ref_lse))
+    with np.errstate(invalid="ignore"):
+        lerr = np.where(both_inf, 0.0, np.abs(lse - ref_lse))
     assert np.nanmax(lerr) <= latol and not np.isnan(lerr).any(), "%s: lse off by %.3g" % (what, np.nanmax(lerr))
 
 
