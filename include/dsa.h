@@ -201,6 +201,33 @@ DSA_API int32_t dsa_debug_kept_indices(const dsa_problem *problem, const dsa_dia
                                int32_t *idx_out, int32_t *count_out, int32_t max_kept,
                                void *stream);
 
+/*
+ * The attention calls above for callers that cannot hand over a workspace.  (The paper has no
+ * counterpart: this is a packaging variant of the two calls, not another method.)
+ *
+ * Who needs it: code that must not allocate device memory at the point of the call -- an
+ * extension running inside a host application's allocation-free section, a latency-critical
+ * serving loop that forbids allocator calls, a process whose device memory was carved up
+ * completely at start-up.  The split-KV partial results go to a fixed DSA_STATIC_SCRATCH_MAX-byte
+ * array inside the library image instead of a caller workspace; the call itself allocates and
+ * frees nothing.  The price: each GPU that loads the library carries those bytes until the
+ * process exits, whether or not this entry point is ever used.
+ *
+ * diag == NULL runs the dense call, otherwise the sparse call; q, caches, out and lse are passed
+ * exactly as above and results are identical to dsa_decode_attention_dense / _sparse.
+ * Problems whose partials exceed the array are refused with DSA_ERR_WORKSPACE_TOO_SMALL and
+ * nothing is launched; dsa_workspace_size() tells the size in advance.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.
+ * All calls share the one array and it keeps whatever the last call left there; nothing in it
+ * needs clearing between calls.  Two calls whose kernels can run at the same time on one GPU
+ * (different streams, different host threads) would overwrite each other's partials: keep calls
+ * of this entry point ordered on one stream per GPU.
+ */
+#define DSA_STATIC_SCRATCH_MAX (8u << 20)
+DSA_API int32_t dsa_decode_attention_static_scratch(const dsa_problem *problem, const dsa_diag_params *diag,
+                                                    void *out, float *lse, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
 
 EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_workspace_size",
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
-           "dsa_combine_splits", "dsa_debug_kept_indices"]
+           "dsa_combine_splits", "dsa_debug_kept_indices",
+           "dsa_decode_attention_static_scratch"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -73,6 +74,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_sparse.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_combine_splits.restype = i32
     lib.dsa_combine_splits.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp]
+    lib.dsa_decode_attention_static_scratch.restype = i32
+    lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
     lib.dsa_debug_kept_indices.restype = i32
     lib.dsa_debug_kept_indices.argtypes = [vp, vp, vp, vp, i32, vp]
     return lib
@@ -233,6 +236,18 @@ def dsa_decode_attention_sparse(problem: Problem, diag: Diag, out: torch.Tensor,
     _check("dsa_decode_attention_sparse",
            _lib.dsa_decode_attention_sparse(_ref(p), _ref(d), _dptr(out), _dptr(lse), _dptr(workspace),
                                             ws_n, _stream(stream)))
+
+
+def dsa_decode_attention_static_scratch(problem: Problem, diag: Optional[Diag], out: torch.Tensor,
+                                        lse: torch.Tensor,
+                                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Dense (diag None) or sparse attention whose split partials use the library's built-in
+    fixed-size scratch array: for callers that may not allocate device memory around the call.
+    Raises DsaError (workspace too small) when the partials would not fit the array."""
+    p = problem.c_struct()
+    d = diag.c_struct() if diag is not None else None
+    _check("dsa_decode_attention_static_scratch",
+           _lib.dsa_decode_attention_static_scratch(_ref(p), _ref(d), _dptr(out), _dptr(lse), _stream(stream)))
 
 
 def dsa_combine_splits(out_part: torch.Tensor, lse_part: torch.Tensor, out: torch.Tensor,

@@ -345,4 +345,37 @@ int32_t dsa_debug_kept_indices(const dsa_problem* problem, const dsa_diag_params
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
+
+// ---- attention without caller-provided scratch ---------------------------------------------------
+// Split-KV partial results normally live in the caller's workspace.  Some callers have nowhere to
+// get one from: code that runs inside a region where device allocation is forbidden (a plugin
+// called under a host framework's "no allocation" section, a real-time loop, a process whose memory
+// pool was handed out completely at start-up).  For them the partials go to this fixed array, which
+// is part of the library image: every GPU that loads the library holds these bytes until exit.
+static __device__ __align__(256) unsigned char g_static_scratch[DSA_STATIC_SCRATCH_MAX];
+
+int32_t dsa_decode_attention_static_scratch(const dsa_problem* problem, const dsa_diag_params* diag, void* out,
+                                            float* lse, void* stream) {
+    // In host code `g_static_scratch` is only a handle for the symbol; the address kernels can use
+    // must be asked for, once per device and with that device current.
+    static void* scratch_addr[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return DSA_ERR_UNSUPPORTED;
+    if (!scratch_addr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        scratch_addr[dev] = ptr;
+    }
+    size_t need = 0;
+    const int32_t rc = dsa_workspace_size(problem, diag, &need);
+    if (rc != DSA_OK) return rc;
+    if (need > DSA_STATIC_SCRATCH_MAX) return DSA_ERR_WORKSPACE_TOO_SMALL;   // problem too large for the fixed array
+    // Nothing in the scratch has to start at zero: every split writes its own lse, and the output of
+    // an empty split is never read, so leftovers of the previous call are harmless.
+    return run_attention(problem, diag, out, lse, scratch_addr[dev], DSA_STATIC_SCRATCH_MAX, stream);
+}
+
 }  // extern "C"
