@@ -55,6 +55,9 @@ def parse_args():
     ap.add_argument("--no-variants", action="store_true", help="skip the dense / other-window timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="also time every configuration (dense and sparse, L2 flushed between calls) "
+                         "and add the table under 'per_config'")
     return ap.parse_args()
 
 
@@ -183,6 +186,68 @@ def time_calls(torch, fn, steps, warmup, sampler=None, barrier=None):
         torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
     return e0.elapsed_time(e1) / 1e3, clocks          # seconds for `steps` calls
+
+
+def time_flushed(torch, fn, flush, iters=30, warmup=3):
+    """Median device time of single calls with the L2 flushed (a 512 MB write) before each."""
+    times = []
+    for i in range(warmup + iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warmup:
+            times.append(e0.elapsed_time(e1) / 1e3)
+    return float(np.median(times)), float(np.min(times))
+
+
+def per_config_table(torch, dsa, synth, dev, peak):
+    """Every configuration, dense and sparse from the same library, one call at a time."""
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    rows = []
+    todo = [(synth.workload(i), None) for i in (1, 2, 3, 4)]
+    for b in (1, 8, 32, 128, 256):
+        todo.append((synth.workload(5, batch=b), [(512, 208), (1024, 416)]))
+    for w, windows in todo:
+        inputs = synth.make_inputs_device(w, dev)
+        host = inputs["host"]
+        prob = dsa.Problem(
+            q=inputs["q"], k_cache=inputs["k_cache"], v_cache=inputs["v_cache"], strides=inputs["strides"],
+            seq_len=inputs["seq_len"], prompt_len=inputs["prompt_len"], num_kv_heads=w.num_kv_heads,
+            max_seq_len=inputs["max_seq_len"], max_prompt_len=w.prompt_len,
+            block_table=inputs["block_table"], block_size=inputs["block_size"],
+            num_blocks=0 if inputs["block_table"] is None else inputs["block_table"].numel())
+        out, lse = dsa.alloc_outputs(prob)
+        ws = dsa.alloc_workspace(prob, None)
+        plan = dsa.dsa_query_plan(prob, None)
+        t_dense, _ = time_flushed(torch, lambda: dsa.dsa_decode_attention_dense(prob, out, lse, ws), flush)
+        b_dense, _ = algorithmic_bytes(w, host, "dense", 0)
+        row = {"config": w.index, "name": w.name, "batch": w.batch,
+               "dense": {"us": round(t_dense * 1e6, 2), "queries_per_sec": round(w.batch / t_dense, 1),
+                         "bytes": b_dense, "GBs": round(b_dense / t_dense / 1e9, 1),
+                         "frac_of_peak": round(b_dense / t_dense / 1e9 / peak, 4),
+                         "n_split": plan.n_split, "launches": plan.launches},
+               "sparse": []}
+        for window, n_att in (windows or [(w.window, w.n_att)]):
+            ww = synth.workload(w.index, batch=w.batch, window=window, n_att=n_att)
+            diag = dsa.Diag(dsa.DSA_MASK_GRID, window, n_att, w.grid_w, w.row_extra)
+            ws2 = dsa.alloc_workspace(prob, diag)
+            plan2 = dsa.dsa_query_plan(prob, diag)
+            t_sp, _ = time_flushed(torch, lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws2), flush)
+            b_sp, _ = algorithmic_bytes(ww, host, "sparse", 0)
+            row["sparse"].append({"window": window, "n_att": n_att, "us": round(t_sp * 1e6, 2),
+                                  "queries_per_sec": round(w.batch / t_sp, 1), "bytes": b_sp,
+                                  "GBs": round(b_sp / t_sp / 1e9, 1),
+                                  "frac_of_peak": round(b_sp / t_sp / 1e9 / peak, 4),
+                                  "speedup_over_dense": round(t_dense / t_sp, 3),
+                                  "ideal_byte_ratio": round(b_dense / b_sp, 3),
+                                  "n_split": plan2.n_split, "launches": plan2.launches})
+        rows.append(row)
+        del inputs, prob, out, lse, ws
+        torch.cuda.empty_cache()
+    return rows
 
 
 def run_ours(args):
@@ -324,6 +389,12 @@ def run_ours(args):
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
+    per_config = None
+    if args.all_configs and rank == 0 and world == 1:
+        del inputs, prob, out, lse
+        torch.cuda.empty_cache()
+        per_config = per_config_table(torch, dsa, synth, dev, peak)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
@@ -340,6 +411,8 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }
+        if per_config is not None:
+            line["per_config"] = per_config
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
