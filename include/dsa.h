@@ -123,7 +123,13 @@ typedef struct dsa_problem {
  *         attended key with the largest (d(o), o).  Same mask for all heads.  (Not in the
  *         paper: a data-free stand-in for its argmin that keeps the diagonals next to the
  *         multiples of the row stride.)
- *   WINDOW nothing skipped (n_att is ignored).
+ *   WINDOW nothing skipped (n_att is ignored).  This is the paper's SlidingWindow baseline.
+ *
+ * Sinks (Section 5.1, the "Diagonal + sink4" variant and the StreamingLLM baseline): the first
+ * n_sink decode tokens are kept at every step in addition to what the mode keeps, and are never
+ * counted against n_att: in steady state n_att + n_sink decode keys are attended.  WINDOW with
+ * n_sink = 4 is StreamingLLM (4 sinks + recent window); GRID or LIST with n_sink = 4 is
+ * Diagonal + sink4 with n_att = budget - 4.
  */
 typedef struct dsa_diag_params {
     int32_t mode;                 /* dsa_mask_mode                                                 */
@@ -134,6 +140,7 @@ typedef struct dsa_diag_params {
     const int32_t *skip_offsets;  /* LIST: device [B, mask_heads, trace_len] int32                 */
     int32_t mask_heads;           /* LIST: 1, H_kv or H_q                                          */
     int32_t trace_len;            /* LIST: entries per trace, >= window - n_att                    */
+    int32_t n_sink;               /* first decode tokens always kept (>= 0; 0 = none)              */
 } dsa_diag_params;
 
 /* What a call will launch (filled by dsa_query_plan; for reporting and for tests). */

@@ -36,6 +36,9 @@
  *   R5  Argmin ties go to the lowest cache index.                       [parity unpinned by the paper]
  *   R6  Attn uses logits sm_scale * q.k, softmax jointly over prompt and kept decode keys;
  *       lse is the natural-log log-sum-exp of those logits.
+ *   R8  Sink variants (Section 5.1, "Diagonal + sink4", StreamingLLM): the first n_sink decode
+ *       tokens are attended at every step on top of what Algorithm 1 attends; the selection runs
+ *       unchanged with its own N_att (callers pass N_att = budget - n_sink).  [parity unpinned]
  *   R7  A request with no decode token yet (seq_len == prompt_len) attends its prompt only; a
  *       request with seq_len == 0 yields out = 0 and lse = -inf.
  *
@@ -276,13 +279,14 @@ int dsa_oracle_combine(const double *out_part, const double *lse_part, int64_t r
  *   mode WINDOW : Algorithm 1 with nothing to skip (N_att = N_r): prompt + the N_r latest tokens
  *   mode GRID   : Algorithm 1, selector ORA_SEL_GRID
  *   mode LIST   : Algorithm 1, selector ORA_SEL_TRACE with the given trace
- * kept_out needs room for L_p + min(p, N_r) entries (L_p + p for DENSE).
+ * plus the first n_sink decode tokens (R8).
+ * kept_out needs room for L_p + min(p, N_r + n_sink) entries (L_p + p for DENSE).
  */
 int dsa_oracle_kept(int32_t mode, int32_t L_p, int32_t p, int32_t N_r, int32_t N_att,
-                    int32_t stride, const int32_t *trace, int32_t trace_len,
+                    int32_t stride, const int32_t *trace, int32_t trace_len, int32_t n_sink,
                     int32_t *kept_out, int32_t *n_kept_out)
 {
-    if (L_p < 0 || p < 0) return ORA_BAD_ARG;
+    if (L_p < 0 || p < 0 || n_sink < 0) return ORA_BAD_ARG;
     int n = 0;
     for (int j = 0; j < L_p; ++j) kept_out[n++] = j;          /* K_p: always attended in full */
     if (p == 0) { *n_kept_out = n; return ORA_OK; }            /* reading R7 */
@@ -303,7 +307,14 @@ int dsa_oracle_kept(int32_t mode, int32_t L_p, int32_t p, int32_t N_r, int32_t N
     else
         rc = ORA_BAD_ARG;
     if (rc == ORA_OK) {
-        for (int i = 0; i < n_idx; ++i) kept_out[n++] = L_p + idx[i];
+        /* sinks: decode tokens 0 .. n_sink-1, attended whether or not idx holds them (R8) */
+        int i = 0;
+        for (int j = 0; j < n_sink && j < p; ++j) {
+            while (i < n_idx && idx[i] < j) kept_out[n++] = L_p + idx[i++];
+            if (i < n_idx && idx[i] == j) ++i;
+            kept_out[n++] = L_p + j;
+        }
+        while (i < n_idx) kept_out[n++] = L_p + idx[i++];
         *n_kept_out = n;
     }
     free(idx);
@@ -330,7 +341,7 @@ int dsa_oracle_decode(int32_t B, int32_t H_q, int32_t H_kv, int32_t D, int32_t d
                       const int32_t *seq_len, const int32_t *prompt_len,
                       const int32_t *block_table, int32_t max_blocks, int32_t block_size,
                       int32_t mode, int32_t N_r, int32_t N_att, int32_t stride_grid,
-                      const int32_t *trace, int32_t mask_heads, int32_t trace_len,
+                      const int32_t *trace, int32_t mask_heads, int32_t trace_len, int32_t n_sink,
                       double sm_scale, double *out, double *lse,
                       int32_t *kept_idx_out, int32_t *kept_cnt_out, int32_t max_kept,
                       int32_t n_threads)
@@ -361,7 +372,7 @@ int dsa_oracle_decode(int32_t B, int32_t H_q, int32_t H_kv, int32_t D, int32_t d
             if (rc == ORA_OK) {
                 const int32_t *tr = (mode == ORA_MODE_LIST && trace)
                     ? trace + ((int64_t)b * mask_heads + mh) * trace_len : NULL;
-                rc = dsa_oracle_kept(mode, L_p, p, N_r, N_att, stride_grid, tr, trace_len, kept, &n_kept);
+                rc = dsa_oracle_kept(mode, L_p, p, N_r, N_att, stride_grid, tr, trace_len, n_sink, kept, &n_kept);
             }
             if (rc == ORA_OK) {
                 for (int i = 0; i < n_kept; ++i) {

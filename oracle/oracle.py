@@ -54,10 +54,10 @@ def lib() -> ctypes.CDLL:
         _lib.dsa_oracle_combine.restype = ctypes.c_int
         _lib.dsa_oracle_combine.argtypes = [vp, vp, i64, i32, i32, vp, vp]
         _lib.dsa_oracle_kept.restype = ctypes.c_int
-        _lib.dsa_oracle_kept.argtypes = [i32, i32, i32, i32, i32, i32, vp, i32, vp, vp]
+        _lib.dsa_oracle_kept.argtypes = [i32, i32, i32, i32, i32, i32, vp, i32, i32, vp, vp]
         _lib.dsa_oracle_decode.restype = ctypes.c_int
         _lib.dsa_oracle_decode.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, i64, i64, i64,
-                                           vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, i32, i32,
+                                           vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, i32, i32, i32,
                                            dbl, vp, vp, vp, vp, i32, i32]
     return _lib
 
@@ -100,12 +100,12 @@ def replay(t: int, n_r: int, n_att: int, selector: int = SEL_TRACE,
 
 
 def kept(mode: int, l_p: int, p: int, n_r: int = 0, n_att: int = 0, stride: int = 0,
-         trace: Optional[Sequence[int]] = None) -> np.ndarray:
+         trace: Optional[Sequence[int]] = None, n_sink: int = 0) -> np.ndarray:
     """Kept cache positions (prompt + attended decode keys) of one request at decode position p."""
     tr = np.ascontiguousarray(np.asarray([] if trace is None else trace, dtype=np.int32))
     outbuf = np.zeros(l_p + p + 1, dtype=np.int32)
     n = ctypes.c_int32(0)
-    rc = lib().dsa_oracle_kept(mode, l_p, p, n_r, n_att, stride, _ptr(tr), len(tr), _ptr(outbuf),
+    rc = lib().dsa_oracle_kept(mode, l_p, p, n_r, n_att, stride, _ptr(tr), len(tr), n_sink, _ptr(outbuf),
                                ctypes.addressof(n))
     _check(rc, "dsa_oracle_kept")
     return outbuf[: n.value].copy()
@@ -158,7 +158,7 @@ def decode(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, seq_len: np.
            prompt_len: np.ndarray, *, num_kv_heads: int, strides: Sequence[int],
            block_table: Optional[np.ndarray] = None, block_size: int = 0,
            mode: int = MODE_DENSE, n_r: int = 0, n_att: int = 0, stride_grid: int = 0,
-           trace: Optional[np.ndarray] = None, sm_scale: Optional[float] = None,
+           trace: Optional[np.ndarray] = None, n_sink: int = 0, sm_scale: Optional[float] = None,
            want_kept: bool = False, n_threads: int = 0):
     """One decode-attention call over a batch.
 
@@ -197,7 +197,7 @@ def decode(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, seq_len: np.
     rc = lib().dsa_oracle_decode(b, h_q, num_kv_heads, d, code, _ptr(q), _ptr(k_cache), _ptr(v_cache),
                                  int(strides[0]), int(strides[1]), int(strides[2]),
                                  _ptr(seq_len), _ptr(prompt_len), _ptr(bt), max_blocks, block_size,
-                                 mode, n_r, n_att, stride_grid, _ptr(tr), mask_heads, trace_len,
+                                 mode, n_r, n_att, stride_grid, _ptr(tr), mask_heads, trace_len, n_sink,
                                  float(sm_scale), _ptr(out), _ptr(lse), _ptr(kept_idx), _ptr(kept_cnt),
                                  max_kept, n_threads)
     _check(rc, "dsa_oracle_decode")

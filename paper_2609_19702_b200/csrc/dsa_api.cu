@@ -123,7 +123,7 @@ int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
     if (!d) return DSA_OK;
     if (d->mode != DSA_MASK_WINDOW && d->mode != DSA_MASK_GRID && d->mode != DSA_MASK_LIST)
         return DSA_ERR_INVALID_ARG;
-    if (d->window < 1) return DSA_ERR_INVALID_ARG;
+    if (d->window < 1 || d->n_sink < 0) return DSA_ERR_INVALID_ARG;
     if (d->mode == DSA_MASK_WINDOW) return DSA_OK;
     if (d->n_att < 1 || d->n_att > d->window) return DSA_ERR_INVALID_ARG;
     if (d->mode == DSA_MASK_GRID) {
@@ -159,7 +159,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         const int64_t lp = p->max_prompt_len > 0 ? p->max_prompt_len : p->max_seq_len;
         int64_t dec = d->window;
         if (pl->mode != MODE_WINDOW) dec = std::min<int64_t>(d->window, (int64_t)d->n_att * (pl->headmask ? G : 1));
-        bound = std::min<int64_t>(bound, lp + dec);
+        bound = std::min<int64_t>(bound, lp + dec + d->n_sink);
     }
     if (bound < 1) bound = 1;
 
@@ -224,6 +224,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.window = d ? d->window : 0;
     a->mask.n_att = d ? (pl.mode == MODE_WINDOW ? d->window : d->n_att) : 0;
     a->mask.stride = (d && pl.mode == MODE_GRID) ? d->grid_w + d->row_extra : 1;
+    a->mask.n_sink = d ? d->n_sink : 0;
     a->mask.skip_offsets = (d && pl.mode == MODE_LIST) ? d->skip_offsets : nullptr;
     a->mask.mask_heads = (d && pl.mode == MODE_LIST) ? d->mask_heads : 1;
     a->mask.trace_len = (d && pl.mode == MODE_LIST) ? d->trace_len : 0;

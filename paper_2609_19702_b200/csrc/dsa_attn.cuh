@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
         }
     };
 
-    if (m.keep_all && r0 >= m.L_p + m.n_win) { write_empty(); return; }
+    if (m.keep_all && r0 >= m.prefix + m.n_win) { write_empty(); return; }
 
     // ---- mask generator -> row list -------------------------------------------------------
     if (a.mask.mode == MODE_LIST && !m.keep_all) {

@@ -8,6 +8,7 @@
 //   window distances  W_t = { 0 .. T },  T = min(t, N_r - 1)
 //   active skips      the first n_act = clamp(t - (N_att - 1), 0, N_r - N_att) selections
 //   kept              prompt [0, L_p)  u  { seq_len - 1 - o : o in W_t \ skips }
+//                     u  the first n_sink decode tokens (attention sinks of the sink variants)
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -21,6 +22,7 @@ struct MaskArgs {
     int window;                // N_r
     int n_att;                 // N_att
     int stride;                // grid_w + row_extra (GRID)
+    int n_sink;                // first decode tokens that are always kept (attention sinks)
     const int* skip_offsets;   // [B, mask_heads, trace_len] (LIST)
     int mask_heads;
     int trace_len;
@@ -35,6 +37,8 @@ struct ReqMask {
     int T;        // largest window distance
     int n_win;    // window candidates = T + 1 (0 when p == 0)
     int w_lo;     // cache position of distance T
+    int prefix;   // positions [0, prefix) are always kept: the prompt and the sinks older than the window
+    int sink_end; // positions below this are sinks or prompt (kept even where the mask skips them)
     int n_act;    // LIST: active skip entries
     int dstar;    // GRID: column distance of the partly kept class (-1: keep none below T)
     int need;     // GRID: how many distances of class dstar are kept (lowest first)
@@ -57,6 +61,7 @@ __device__ __forceinline__ ReqMask req_mask_setup(const MaskArgs& a, int seq_len
     m.L_p = max(0, min(prompt_len, m.S));
     m.p = m.S - m.L_p;
     m.n_act = 0; m.dstar = -1; m.need = 0; m.keep_all = true;
+    m.prefix = m.L_p; m.sink_end = m.L_p;
     if (a.mode == MODE_DENSE) {
         m.T = m.p - 1; m.n_win = m.p; m.w_lo = m.L_p;
         return m;
@@ -65,6 +70,8 @@ __device__ __forceinline__ ReqMask req_mask_setup(const MaskArgs& a, int seq_len
     m.T = min(t, a.window - 1);
     m.n_win = m.p > 0 ? m.T + 1 : 0;
     m.w_lo = m.S - m.n_win;
+    m.sink_end = m.L_p + min(a.n_sink, m.p);
+    m.prefix = min(m.sink_end, m.w_lo);
     if (a.mode == MODE_WINDOW || m.p == 0 || t < a.n_att - 1) return m;   // phase 1 / nothing to skip
     if (a.mode == MODE_LIST) {
         m.n_act = min(min(t - (a.n_att - 1), a.window - a.n_att), a.trace_len);
@@ -154,32 +161,36 @@ __device__ __forceinline__ int enumerate_kept(const MaskArgs& a, const ReqMask& 
                                               const unsigned* bitmaps, int r0, int r1,
                                               int* s_warp, Sink sink) {
     constexpr unsigned ALL = (1u << SLOTS) - 1u;
-    // the prompt: always attended in full
-    for (int r = max(r0, 0) + (int)threadIdx.x; r < min(r1, m.L_p); r += NT) sink(r - r0, r, ALL);
+    // the prompt (always attended in full) and the sinks that have left the window
+    for (int r = max(r0, 0) + (int)threadIdx.x; r < min(r1, m.prefix); r += NT) sink(r - r0, r, ALL);
     if (m.keep_all) {
-        // contiguous window: rank L_p + c  <->  position w_lo + c
-        const int lo = max(r0, m.L_p), hi = min(r1, m.L_p + m.n_win);
-        for (int r = lo + (int)threadIdx.x; r < hi; r += NT) sink(r - r0, m.w_lo + (r - m.L_p), ALL);
-        return m.L_p + m.n_win;
+        // contiguous window: rank prefix + c  <->  position w_lo + c
+        const int lo = max(r0, m.prefix), hi = min(r1, m.prefix + m.n_win);
+        for (int r = lo + (int)threadIdx.x; r < hi; r += NT) sink(r - r0, m.w_lo + (r - m.prefix), ALL);
+        return m.prefix + m.n_win;
     }
     // Each thread owns a contiguous run of window candidates (ascending position = descending
     // distance): count, scan, then emit.
     const int per = (m.n_win + NT - 1) / NT;
     const int c0 = min((int)threadIdx.x * per, m.n_win), c1 = min(c0 + per, m.n_win);
+    // a sink that is still inside the window is kept whatever the mask says
+    auto bits_at = [&](int c) -> unsigned {
+        return (m.w_lo + c < m.sink_end) ? ALL : keep_bits<SLOTS>(a, m, bitmaps, m.T - c);
+    };
     int cnt = 0;
-    for (int c = c0; c < c1; ++c) cnt += keep_bits<SLOTS>(a, m, bitmaps, m.T - c) != 0u;
+    for (int c = c0; c < c1; ++c) cnt += bits_at(c) != 0u;
     int total;
-    int rank = m.L_p + block_excl_scan<NT>(cnt, total, s_warp);
+    int rank = m.prefix + block_excl_scan<NT>(cnt, total, s_warp);
     if (rank < r1 && rank + cnt > r0) {
         for (int c = c0; c < c1; ++c) {
-            const unsigned bits = keep_bits<SLOTS>(a, m, bitmaps, m.T - c);
+            const unsigned bits = bits_at(c);
             if (bits) {
                 if (rank >= r0 && rank < r1) sink(rank - r0, m.w_lo + c, bits);
                 ++rank;
             }
         }
     }
-    return m.L_p + total;
+    return m.prefix + total;
 }
 
 }  // namespace dsa

@@ -62,12 +62,25 @@ def _check_all_modes(dsa, inp, *, f32=False, split_tokens=0, list_heads=(1,), se
     idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, s_max)
     util.assert_kept_equal(idx, cnt, ref, what + " grid")
 
+    # sink variants: StreamingLLM (window + sinks) and Diagonal + sink4
+    for mode_gpu, mode_ora, tag in ((dsa.DSA_MASK_WINDOW, ora.MODE_WINDOW, "streaming"),
+                                    (dsa.DSA_MASK_GRID, ora.MODE_GRID, "grid+sink")):
+        diag = dsa.Diag(mode_gpu, w.window, w.n_att, w.grid_w, w.row_extra, n_sink=4)
+        ref = util.oracle_run(inp, mode_ora, n_r=w.window, n_att=w.n_att, stride=w.stride, n_sink=4,
+                              want_kept=True)
+        out, lse = _run_gpu(dsa, prob, diag)
+        util.assert_close(out, lse, ref, f32, what + " " + tag)
+        idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, s_max)
+        util.assert_kept_equal(idx, cnt, ref, what + " " + tag)
+
     rng = np.random.default_rng(1000 + seed)
     for mh in list_heads:
         trace = synth.random_valid_trace(rng, w.window, w.n_att, (w.batch, mh))
+        n_sink = 4 if mh == list_heads[-1] else 0
         diag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att,
-                        skip_offsets=torch.from_numpy(trace).cuda())
-        ref = util.oracle_run(inp, ora.MODE_LIST, n_r=w.window, n_att=w.n_att, trace=trace, want_kept=True)
+                        skip_offsets=torch.from_numpy(trace).cuda(), n_sink=n_sink)
+        ref = util.oracle_run(inp, ora.MODE_LIST, n_r=w.window, n_att=w.n_att, trace=trace, n_sink=n_sink,
+                              want_kept=True)
         out, lse = _run_gpu(dsa, prob, diag)
         util.assert_close(out, lse, ref, f32, what + " list mh=%d" % mh)
         idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, s_max)

@@ -166,6 +166,31 @@ def test_kept_positions_modes():
     assert ora.kept(ora.MODE_WINDOW, 4, 9, 9, 9).tolist() == list(range(13))
 
 
+def test_sink_variants_against_set_arithmetic():
+    # Section 5.1: StreamingLLM = 4 sinks (first decode tokens) + recent window, prompt always kept;
+    # Diagonal + sink4 = the same sinks on top of the diagonal selection
+    l_p, n_r, n_att, stride, n_sink = 6, 12, 5, 4, 4
+    rng = np.random.default_rng(11)
+    trace = synth.random_valid_trace(rng, n_r, n_att).tolist()
+    for p in range(0, 40):
+        t = p - 1
+        sinks = {l_p + j for j in range(min(n_sink, p))}
+        prompt = set(range(l_p))
+        win = ora.kept(ora.MODE_WINDOW, l_p, p, n_r, n_r, n_sink=n_sink)
+        want = prompt | sinks | set(range(l_p + max(0, p - n_r), l_p + p))
+        assert win.tolist() == sorted(want)
+        grid = ora.kept(ora.MODE_GRID, l_p, p, n_r, n_att, stride, n_sink=n_sink)
+        base = {l_p + t - o for o in brute.kept_offsets_grid(t, n_r, n_att, stride)} if p else set()
+        assert grid.tolist() == sorted(prompt | sinks | base)
+        lst = ora.kept(ora.MODE_LIST, l_p, p, n_r, n_att, trace=trace, n_sink=n_sink)
+        base = {l_p + t - o for o in brute.kept_offsets_from_trace(t, n_r, n_att, trace)} if p else set()
+        assert lst.tolist() == sorted(prompt | sinks | base)
+        if p >= n_r + n_sink:                       # sinks have left the window: budget is exact
+            assert len(grid) == l_p + n_att + n_sink and len(lst) == l_p + n_att + n_sink
+    assert ora.kept(ora.MODE_GRID, l_p, 9, n_r, n_att, stride, n_sink=0).tolist() == \
+        ora.kept(ora.MODE_GRID, l_p, 9, n_r, n_att, stride).tolist()
+
+
 def test_cost_model_ratio_last_step():
     # Section 4 cost analysis: per-step compute shrinks by (L_dec + L_p) / (N_att + L_p)
     for l_dec, l_p, sparsity in ((576, 50, 0.95), (1024, 50, 0.90)):

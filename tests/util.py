@@ -12,7 +12,7 @@ OUT_ATOL, OUT_RTOL, LSE_ATOL = 1e-2, 1e-2, 1e-3
 F32_ATOL, F32_RTOL, F32_LSE_ATOL = 2e-5, 2e-5, 2e-5
 
 
-def oracle_run(inp, mode, *, n_r=0, n_att=0, stride=0, trace=None, want_kept=False, requests=None):
+def oracle_run(inp, mode, *, n_r=0, n_att=0, stride=0, trace=None, n_sink=0, want_kept=False, requests=None):
     """Oracle on a host batch (optionally on a subset of requests)."""
     w = inp["workload"]
     q, seq, pl, bt = inp["q"], inp["seq_len"], inp["prompt_len"], inp["block_table"]
@@ -27,7 +27,7 @@ def oracle_run(inp, mode, *, n_r=0, n_att=0, stride=0, trace=None, want_kept=Fal
             trace = trace[req]
     return ora.decode(q, inp["k_cache"], inp["v_cache"], seq, pl, num_kv_heads=w.num_kv_heads,
                       strides=inp["strides"], block_table=bt, block_size=inp["block_size"],
-                      mode=mode, n_r=n_r, n_att=n_att, stride_grid=stride, trace=trace,
+                      mode=mode, n_r=n_r, n_att=n_att, stride_grid=stride, trace=trace, n_sink=n_sink,
                       want_kept=want_kept)
 
 
