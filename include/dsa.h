@@ -125,6 +125,15 @@ typedef struct dsa_problem {
  *         multiples of the row stride.)
  *   WINDOW nothing skipped (n_att is ignored).  This is the paper's SlidingWindow baseline.
  *
+ * Selection (Algorithm 1, phase 2: "select newly skipped KV", fused into the attention pass as
+ * in Section 5.1).  With `select` set, a request whose step t lies in N_att-1 .. N_r-2 also gets
+ * the next trace entry: among the decode keys it attends (sinks excluded) the one with the lowest
+ * softmax weight -- the lowest logit; equal logits go to the lowest cache index -- is found per
+ * query head and its distance is written to skip_offsets[b][h][t - (N_att-1)], which takes effect
+ * from the next step on.  Calling the sparse call once per decode step with the same buffer thus
+ * grows the trace exactly as Algorithm 1 grows skip_idx.  Entries are decided on float32 logits;
+ * -1 is written if there is no candidate.  Requests outside those steps are left untouched.
+ *
  * Sinks (Section 5.1, the "Diagonal + sink4" variant and the StreamingLLM baseline): the first
  * n_sink decode tokens are kept at every step in addition to what the mode keeps, and are never
  * counted against n_att: in steady state n_att + n_sink decode keys are attended.  WINDOW with
@@ -137,10 +146,12 @@ typedef struct dsa_diag_params {
     int32_t n_att;                /* N_att, 1 <= n_att <= window                                   */
     int32_t grid_w;               /* GRID: image tokens per row                                    */
     int32_t row_extra;            /* GRID: row-end / separator tokens per row (>= 0)               */
-    const int32_t *skip_offsets;  /* LIST: device [B, mask_heads, trace_len] int32                 */
+    int32_t *skip_offsets;        /* LIST: device [B, mask_heads, trace_len] int32 (written when   */
+                                  /* `select` is set, otherwise only read)                         */
     int32_t mask_heads;           /* LIST: 1, H_kv or H_q                                          */
     int32_t trace_len;            /* LIST: entries per trace, >= window - n_att                    */
     int32_t n_sink;               /* first decode tokens always kept (>= 0; 0 = none)              */
+    int32_t select;               /* LIST, mask_heads == H_q: also run the phase-2 selection       */
 } dsa_diag_params;
 
 /* What a call will launch (filled by dsa_query_plan; for reporting and for tests). */

@@ -38,7 +38,9 @@
  *       lse is the natural-log log-sum-exp of those logits.
  *   R8  Sink variants (Section 5.1, "Diagonal + sink4", StreamingLLM): the first n_sink decode
  *       tokens are attended at every step on top of what Algorithm 1 attends; the selection runs
- *       unchanged with its own N_att (callers pass N_att = budget - n_sink).  [parity unpinned]
+ *       unchanged with its own N_att (callers pass N_att = budget - n_sink), except that a sink
+ *       is never a candidate of the argmin ("diagonal selection for the remaining slots").
+ *                                                                        [parity unpinned]
  *   R7  A request with no decode token yet (seq_len == prompt_len) attends its prompt only; a
  *       request with seq_len == 0 yields out = 0 and lse = -inf.
  *
@@ -59,7 +61,7 @@
 #define ORA_NO_MEM (-3)
 
 enum { ORA_F64 = 0, ORA_F32 = 1, ORA_BF16 = 2 };
-enum { ORA_SEL_TRACE = 0, ORA_SEL_GRID = 1 };
+enum { ORA_SEL_TRACE = 0, ORA_SEL_GRID = 1, ORA_SEL_ARGMIN = 2 };
 enum { ORA_MODE_DENSE = 0, ORA_MODE_WINDOW = 1, ORA_MODE_GRID = 2, ORA_MODE_LIST = 3 };
 
 static double load_elem(const void *base, int dtype, int64_t i)
@@ -82,6 +84,22 @@ int dsa_oracle_num_threads(void)
 #endif
 }
 
+int dsa_oracle_select_argmin(const void *q_row, const void *k_base, int dtype,
+                             const int64_t *k_rows, int32_t n_idx, int32_t D, double sm_scale,
+                             int32_t *j_star, double *w_out);
+
+/* what the argmin selector needs: the query of every step and the decode keys */
+typedef struct {
+    const void *q_steps;      /* query of step t starts at element t * q_step_stride */
+    int64_t q_step_stride;
+    const void *k_base;
+    const int64_t *k_rows;    /* element offset of decode key j */
+    int dtype;
+    int32_t D;
+    double sm_scale;
+    int32_t n_sink;           /* decode keys 0 .. n_sink-1 are sinks: never candidates (R8) */
+} argmin_ctx;
+
 /* column distance on the raster grid of a key o tokens behind the query (reading R4) */
 static int grid_col_dist(int o, int stride)
 {
@@ -102,14 +120,16 @@ static int grid_col_dist(int o, int stride)
  *   skip_out  [>= N_r]     : skip_idx as it stands at the END of step t_final (after an append)
  * Returns ORA_OK, ORA_BAD_ARG, ORA_BAD_TRACE (trace too short, or names a key not in idx).
  */
-int dsa_oracle_replay(int32_t t_final, int32_t N_r, int32_t N_att, int32_t selector,
-                      const int32_t *trace, int32_t trace_len, int32_t stride,
-                      int32_t *idx_out, int32_t *n_idx_out,
-                      int32_t *skip_out, int32_t *n_skip_out)
+static int replay_core(int32_t t_final, int32_t N_r, int32_t N_att, int32_t selector,
+                       const int32_t *trace, int32_t trace_len, int32_t stride, const argmin_ctx *ctx,
+                       int32_t *idx_out, int32_t *n_idx_out,
+                       int32_t *skip_out, int32_t *n_skip_out,
+                       int32_t *trace_out, int32_t *n_trace_out)
 {
     if (t_final < 0 || N_att < 1 || N_r < N_att) return ORA_BAD_ARG;
     if (selector == ORA_SEL_GRID && stride < 1) return ORA_BAD_ARG;
-    if (selector != ORA_SEL_GRID && selector != ORA_SEL_TRACE) return ORA_BAD_ARG;
+    if (selector != ORA_SEL_GRID && selector != ORA_SEL_TRACE && selector != ORA_SEL_ARGMIN) return ORA_BAD_ARG;
+    if (selector == ORA_SEL_ARGMIN && (!ctx || ctx->n_sink >= N_att)) return ORA_BAD_ARG;
 
     int32_t *skip_idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(N_r + 1));
     int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(N_r + 1));
@@ -150,6 +170,22 @@ int dsa_oracle_replay(int32_t t_final, int32_t N_r, int32_t N_att, int32_t selec
                     int32_t want = t - trace[n_sel];
                     for (int i = 0; i < n_idx; ++i) if (idx[i] == want) chosen = want;
                     if (chosen < 0) { rc = ORA_BAD_TRACE; break; }
+                } else if (selector == ORA_SEL_ARGMIN) {
+                    /* w <- softmax(Q_t . K[idx]^T); j* <- argmin_j w[j]   (sinks are not in the race) */
+                    int64_t *rows = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n_idx + 1));
+                    int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_idx + 1));
+                    if (!rows || !cand) { free(rows); free(cand); rc = ORA_NO_MEM; break; }
+                    int n_cand = 0;
+                    for (int i = 0; i < n_idx; ++i)
+                        if (idx[i] >= ctx->n_sink) { cand[n_cand] = idx[i]; rows[n_cand++] = ctx->k_rows[idx[i]]; }
+                    int32_t j_star = -1;
+                    size_t esz = ctx->dtype == ORA_F64 ? 8 : (ctx->dtype == ORA_F32 ? 4 : 2);
+                    const void *q_t = (const char *)ctx->q_steps + (size_t)t * (size_t)ctx->q_step_stride * esz;
+                    rc = dsa_oracle_select_argmin(q_t, ctx->k_base, ctx->dtype, rows, n_cand, ctx->D,
+                                                  ctx->sm_scale, &j_star, NULL);
+                    if (rc == ORA_OK) chosen = cand[j_star];
+                    free(rows); free(cand);
+                    if (rc != ORA_OK) break;
                 } else {
                     int best_d = -1, best_o = -1;
                     for (int i = 0; i < n_idx; ++i) {
@@ -162,6 +198,7 @@ int dsa_oracle_replay(int32_t t_final, int32_t N_r, int32_t N_att, int32_t selec
                 }
                 skip_idx[n_skip++] = chosen;              /* skip_idx.append(idx[j*]) */
                 in_skip[chosen] = 1;
+                if (trace_out) trace_out[n_sel] = t - chosen;   /* the same choice as a distance */
                 ++n_sel;
             }
         }
@@ -171,9 +208,39 @@ int dsa_oracle_replay(int32_t t_final, int32_t N_r, int32_t N_att, int32_t selec
         *n_idx_out = n_idx;
         if (skip_out) for (int i = 0; i < n_skip; ++i) skip_out[i] = skip_idx[i];
         if (n_skip_out) *n_skip_out = n_skip;
+        if (n_trace_out) *n_trace_out = n_sel;
     }
     free(skip_idx); free(idx); free(present); free(in_skip);
     return rc;
+}
+
+int dsa_oracle_replay(int32_t t_final, int32_t N_r, int32_t N_att, int32_t selector,
+                      const int32_t *trace, int32_t trace_len, int32_t stride,
+                      int32_t *idx_out, int32_t *n_idx_out,
+                      int32_t *skip_out, int32_t *n_skip_out)
+{
+    if (selector == ORA_SEL_ARGMIN) return ORA_BAD_ARG;
+    return replay_core(t_final, N_r, N_att, selector, trace, trace_len, stride, NULL,
+                       idx_out, n_idx_out, skip_out, n_skip_out, NULL, NULL);
+}
+
+/*
+ * Algorithm 1 with its own selection rule (phase 2: softmax over the attended decode keys,
+ * argmin), for one head of one sequence: runs steps 0 .. t_final with query q_steps[t] at step t
+ * and decode key j at k_rows[j].  Returns what step t_final attends (idx_out, decode-relative)
+ * and every selection made so far as distances behind the query of its step (trace_out, in
+ * selection order) -- the form in which the attention calls take a trace.
+ */
+int dsa_oracle_replay_argmin(int32_t t_final, int32_t N_r, int32_t N_att, int32_t n_sink,
+                             const void *q_steps, int64_t q_step_stride,
+                             const void *k_base, int dtype, const int64_t *k_rows,
+                             int32_t D, double sm_scale,
+                             int32_t *idx_out, int32_t *n_idx_out,
+                             int32_t *trace_out, int32_t *n_trace_out)
+{
+    argmin_ctx ctx = { q_steps, q_step_stride, k_base, k_rows, dtype, D, sm_scale, n_sink };
+    return replay_core(t_final, N_r, N_att, ORA_SEL_ARGMIN, NULL, 0, 0, &ctx,
+                       idx_out, n_idx_out, NULL, NULL, trace_out, n_trace_out);
 }
 
 /*

@@ -21,7 +21,7 @@ _SRC = os.path.join(_HERE, "dsa_oracle.c")
 _LIB = os.path.join(_HERE, "libdsa_oracle.so")
 
 F64, F32, BF16 = 0, 1, 2
-SEL_TRACE, SEL_GRID = 0, 1
+SEL_TRACE, SEL_GRID, SEL_ARGMIN = 0, 1, 2
 MODE_DENSE, MODE_WINDOW, MODE_GRID, MODE_LIST = 0, 1, 2, 3
 
 _lib = None
@@ -47,6 +47,9 @@ def lib() -> ctypes.CDLL:
         _lib.dsa_oracle_num_threads.restype = ctypes.c_int
         _lib.dsa_oracle_replay.restype = ctypes.c_int
         _lib.dsa_oracle_replay.argtypes = [i32, i32, i32, i32, vp, i32, i32, vp, vp, vp, vp]
+        _lib.dsa_oracle_replay_argmin.restype = ctypes.c_int
+        _lib.dsa_oracle_replay_argmin.argtypes = [i32, i32, i32, i32, vp, i64, vp, ctypes.c_int, vp, i32, dbl,
+                                                  vp, vp, vp, vp]
         _lib.dsa_oracle_select_argmin.restype = ctypes.c_int
         _lib.dsa_oracle_select_argmin.argtypes = [vp, vp, ctypes.c_int, vp, i32, i32, dbl, vp, vp]
         _lib.dsa_oracle_attend.restype = ctypes.c_int
@@ -97,6 +100,25 @@ def replay(t: int, n_r: int, n_att: int, selector: int = SEL_TRACE,
                                  ctypes.addressof(n_idx), _ptr(skip), ctypes.addressof(n_skip))
     _check(rc, "dsa_oracle_replay")
     return idx[: n_idx.value].copy(), skip[: n_skip.value].copy()
+
+
+def replay_argmin(t: int, n_r: int, n_att: int, q_steps: np.ndarray, q_step_stride: int, k: np.ndarray,
+                  k_rows: np.ndarray, d: int, sm_scale: float, n_sink: int = 0):
+    """Algorithm 1 with its argmin selection for one head: query of step s at element
+    ``s * q_step_stride`` of ``q_steps``, decode key j at element ``k_rows[j]`` of ``k``.
+    Returns (idx attended at step t, trace of distances selected so far)."""
+    assert q_steps.flags.c_contiguous and k.flags.c_contiguous
+    assert _dtype_code(q_steps) == _dtype_code(k)
+    rows = np.ascontiguousarray(k_rows, dtype=np.int64)
+    idx = np.zeros(n_r + 1, dtype=np.int32)
+    tr = np.zeros(max(n_r - n_att, 1), dtype=np.int32)
+    n_idx = ctypes.c_int32(0)
+    n_tr = ctypes.c_int32(0)
+    rc = lib().dsa_oracle_replay_argmin(t, n_r, n_att, n_sink, _ptr(q_steps), int(q_step_stride), _ptr(k),
+                                        _dtype_code(k), _ptr(rows), d, float(sm_scale), _ptr(idx),
+                                        ctypes.addressof(n_idx), _ptr(tr), ctypes.addressof(n_tr))
+    _check(rc, "dsa_oracle_replay_argmin")
+    return idx[: n_idx.value].copy(), tr[: n_tr.value].copy()
 
 
 def kept(mode: int, l_p: int, p: int, n_r: int = 0, n_att: int = 0, stride: int = 0,

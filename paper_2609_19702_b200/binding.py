@@ -44,7 +44,8 @@ class dsa_diag_params(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("window", ctypes.c_int32), ("n_att", ctypes.c_int32),
                 ("grid_w", ctypes.c_int32), ("row_extra", ctypes.c_int32),
                 ("skip_offsets", ctypes.c_void_p), ("mask_heads", ctypes.c_int32),
-                ("trace_len", ctypes.c_int32), ("n_sink", ctypes.c_int32)]
+                ("trace_len", ctypes.c_int32), ("n_sink", ctypes.c_int32),
+                ("select", ctypes.c_int32)]
 
 
 class dsa_plan_info(ctypes.Structure):
@@ -167,12 +168,14 @@ class Diag:
     row_extra: int = 0
     skip_offsets: Optional[torch.Tensor] = None   # int32 [B, mask_heads, trace_len] (LIST)
     n_sink: int = 0
+    select: bool = False                          # LIST: also append the next trace entry (in place)
 
     def c_struct(self) -> dsa_diag_params:
         d = dsa_diag_params()
         d.mode, d.window, d.n_att = self.mode, self.window, self.n_att
         d.grid_w, d.row_extra = self.grid_w, self.row_extra
         d.n_sink = self.n_sink
+        d.select = 1 if self.select else 0
         if self.skip_offsets is not None:
             t = self.skip_offsets
             assert t.dtype == torch.int32 and t.is_contiguous() and t.dim() == 3

@@ -28,38 +28,38 @@ struct Plan {
     int mode;            // MODE_*
     int G;
     bool headmask;
+    bool select;
     int tile, stages;
     int chunk, n_split;
     int bitmap_words;
     int64_t grid;
     size_t smem;
-    size_t ws_out_bytes, ws_total;
+    size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
 };
 
-template <typename T, int D, int G, bool HM>
+template <typename T, int D, int G, bool HM, bool SEL>
 struct KernelPick {
     // Small tiles (2 KB of K + 2 KB of V) in a 4-deep ring: 16-20 KB of shared memory per block, so
     // 8 or more blocks share an SM and their start-up and merge phases overlap each other's
     // streaming.  (Measured on the paged batch-256 workload: 32-row tiles with 3 blocks/SM reach
     // 5.7 TB/s, these reach 6.6 TB/s; the dense call is flat at 7.2 TB/s either way.)
     // -DDSA_TUNE_TILE / -DDSA_TUNE_STAGES override the bf16, head_dim 128 choice in tuning builds.
-    static constexpr bool kMain = sizeof(T) == 2 && D == 128;
     static constexpr int kTileDefault = 2048 / (D * (int)sizeof(T));
     static constexpr int kStagesDefault = 4;
 #ifdef DSA_TUNE_TILE
-    static constexpr int TILE = kMain ? DSA_TUNE_TILE : kTileDefault;
+    static constexpr int TILE = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_TILE : kTileDefault;
 #else
     static constexpr int TILE = kTileDefault;
 #endif
 #ifdef DSA_TUNE_STAGES
-    static constexpr int STAGES = kMain ? DSA_TUNE_STAGES : kStagesDefault;
+    static constexpr int STAGES = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_STAGES : kStagesDefault;
 #else
     static constexpr int STAGES = kStagesDefault;
 #endif
-    using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM>;
+    using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM, SEL>;
     static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM>;
+        auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
         static bool configured[kMaxDevices] = {};
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -74,16 +74,20 @@ struct KernelPick {
     }
 };
 
-// Dispatch over (dtype, head_dim, group size, per-head masks).  F(KernelPick<...>) -> R.
+// Dispatch over (dtype, head_dim, group size, per-head masks, fused selection).  Selection needs one
+// mask per query head, so it comes with per-head masks whenever the group is larger than one.
 template <class F>
-int32_t dispatch(int dtype, int D, int G, bool hm, F&& f) {
-#define DSA_CASE_G(T, DD)                                                                     \
-    switch (G) {                                                                              \
-        case 1: return f(KernelPick<T, DD, 1, false>{});                                      \
-        case 2: return hm ? f(KernelPick<T, DD, 2, true>{}) : f(KernelPick<T, DD, 2, false>{}); \
-        case 4: return hm ? f(KernelPick<T, DD, 4, true>{}) : f(KernelPick<T, DD, 4, false>{}); \
-        case 8: return hm ? f(KernelPick<T, DD, 8, true>{}) : f(KernelPick<T, DD, 8, false>{}); \
-        default: return DSA_ERR_UNSUPPORTED;                                                  \
+int32_t dispatch(int dtype, int D, int G, bool hm, bool sel, F&& f) {
+#define DSA_CASE_HM(T, DD, GG)                                                         \
+    if (sel) return f(KernelPick<T, DD, GG, (GG > 1), true>{});                        \
+    return hm ? f(KernelPick<T, DD, GG, (GG > 1), false>{}) : f(KernelPick<T, DD, GG, false, false>{});
+#define DSA_CASE_G(T, DD)                         \
+    switch (G) {                                  \
+        case 1: { DSA_CASE_HM(T, DD, 1) }         \
+        case 2: { DSA_CASE_HM(T, DD, 2) }         \
+        case 4: { DSA_CASE_HM(T, DD, 4) }         \
+        case 8: { DSA_CASE_HM(T, DD, 8) }         \
+        default: return DSA_ERR_UNSUPPORTED;      \
     }
     if (dtype == DSA_BF16) {
         if (D == 64) { DSA_CASE_G(__nv_bfloat16, 64) }
@@ -93,6 +97,7 @@ int32_t dispatch(int dtype, int D, int G, bool hm, F&& f) {
         if (D == 128) { DSA_CASE_G(float, 128) }
     }
 #undef DSA_CASE_G
+#undef DSA_CASE_HM
     return DSA_ERR_UNSUPPORTED;
 }
 
@@ -135,6 +140,8 @@ int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
         return DSA_ERR_INVALID_ARG;
     if (d->trace_len < d->window - d->n_att) return DSA_ERR_INVALID_ARG;
     if (d->window - d->n_att > 0 && p->batch > 0 && !d->skip_offsets) return DSA_ERR_INVALID_ARG;
+    if (d->select && d->mask_heads != p->num_q_heads) return DSA_ERR_UNSUPPORTED;   // one selection per attention head
+    if (d->select && d->n_sink >= d->n_att) return DSA_ERR_INVALID_ARG;             // no candidate would be left
     return DSA_OK;
 }
 
@@ -152,6 +159,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     // per-query-head masks inside a group: rows of the union are read, heads mask individually
     pl->headmask = pl->mode == MODE_LIST && G > 1 && d->mask_heads == p->num_q_heads;
     pl->bitmap_words = pl->mode == MODE_LIST ? (d->window + 31) / 32 : 0;
+    pl->select = pl->mode == MODE_LIST && d->select != 0;
 
     // upper bound of kept rows per (request, kv head)
     int64_t bound = p->max_seq_len;
@@ -164,7 +172,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     if (bound < 1) bound = 1;
 
     size_t smem_probe = 0;
-    rc = dispatch(p->dtype, p->head_dim, G, pl->headmask, [&](auto pick) -> int32_t {
+    rc = dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
         pl->tile = P::TILE;
         pl->stages = P::STAGES;
@@ -191,7 +199,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->grid = (int64_t)p->batch * p->num_kv_heads * pl->n_split;
     if (pl->grid > 0x7fffffffLL) return DSA_ERR_UNSUPPORTED;
 
-    dispatch(p->dtype, p->head_dim, G, pl->headmask, [&](auto pick) -> int32_t {
+    dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
         smem_probe = P::smem(pl->chunk, pl->bitmap_words);
         return DSA_OK;
@@ -202,9 +210,13 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     if (pl->n_split > 1) {
         const size_t rows = (size_t)p->batch * p->num_q_heads * pl->n_split;
         pl->ws_out_bytes = (rows * p->head_dim * sizeof(float) + 255) / 256 * 256;
-        pl->ws_total = pl->ws_out_bytes + (rows * sizeof(float) + 255) / 256 * 256;
+        pl->ws_lse_bytes = (rows * sizeof(float) + 255) / 256 * 256;
+        // selection candidates per split (logit, distance) and the trace entry per (request, head)
+        pl->ws_sel_bytes = pl->select ? pl->ws_lse_bytes : 0;
+        const size_t k_bytes = pl->select ? ((size_t)p->batch * p->num_q_heads * sizeof(int) + 255) / 256 * 256 : 0;
+        pl->ws_total = pl->ws_out_bytes + pl->ws_lse_bytes + 2 * pl->ws_sel_bytes + k_bytes;
     } else {
-        pl->ws_out_bytes = 0;
+        pl->ws_out_bytes = pl->ws_lse_bytes = pl->ws_sel_bytes = 0;
         pl->ws_total = 0;
     }
     return DSA_OK;
@@ -226,20 +238,26 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.stride = (d && pl.mode == MODE_GRID) ? d->grid_w + d->row_extra : 1;
     a->mask.n_sink = d ? d->n_sink : 0;
     a->mask.skip_offsets = (d && pl.mode == MODE_LIST) ? d->skip_offsets : nullptr;
+    a->mask.select = pl.select ? 1 : 0;
     a->mask.mask_heads = (d && pl.mode == MODE_LIST) ? d->mask_heads : 1;
     a->mask.trace_len = (d && pl.mode == MODE_LIST) ? d->trace_len : 0;
     a->mask.bitmap_words = pl.bitmap_words;
     a->chunk = pl.chunk; a->n_split = pl.n_split;
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
+    a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
 }
 
 int32_t launch_combine(const float* out_part, const float* lse_part, int64_t rows, int D, int n_split,
-                       void* out, float* lse, int dtype, cudaStream_t st) {
+                       void* out, float* lse, int dtype, cudaStream_t st, const float* sel_val = nullptr,
+                       const int* sel_off = nullptr, const int* sel_k = nullptr, int* trace = nullptr,
+                       int trace_len = 0) {
     if (rows == 0) return DSA_OK;
     if (dtype == DSA_BF16)
-        dsa_combine_kernel<__nv_bfloat16><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse);
+        dsa_combine_kernel<__nv_bfloat16><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse,
+                                                                      sel_val, sel_off, sel_k, trace, trace_len);
     else
-        dsa_combine_kernel<float><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse);
+        dsa_combine_kernel<float><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse,
+                                                              sel_val, sel_off, sel_k, trace, trace_len);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
@@ -259,13 +277,19 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     fill_args(p, d, pl, &a);
     if (pl.n_split > 1) {
         a.out_part = reinterpret_cast<float*>(workspace);
-        a.lse_part = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + pl.ws_out_bytes);
+        unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
+        a.lse_part = reinterpret_cast<float*>(ws + pl.ws_out_bytes);
+        if (pl.select) {
+            a.sel_val_part = reinterpret_cast<float*>(ws + pl.ws_out_bytes + pl.ws_lse_bytes);
+            a.sel_off_part = reinterpret_cast<int*>(ws + pl.ws_out_bytes + pl.ws_lse_bytes + pl.ws_sel_bytes);
+            a.sel_k = reinterpret_cast<int*>(ws + pl.ws_out_bytes + pl.ws_lse_bytes + 2 * pl.ws_sel_bytes);
+        }
     } else {
         a.out = out; a.lse = lse;
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, [&](auto pick) -> int32_t {
+    rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, pl.select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
         err = P::launch(a, pl.grid, pl.smem, st);
         return DSA_OK;
@@ -274,7 +298,8 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     if (err != cudaSuccess) return cuda_fail(err);
     if (pl.n_split > 1)
         return launch_combine(a.out_part, a.lse_part, (int64_t)p->batch * p->num_q_heads, p->head_dim,
-                              pl.n_split, out, lse, p->dtype, st);
+                              pl.n_split, out, lse, p->dtype, st, a.sel_val_part, a.sel_off_part, a.sel_k,
+                              pl.select ? d->skip_offsets : nullptr, pl.select ? d->trace_len : 0);
     return DSA_OK;
 }
 

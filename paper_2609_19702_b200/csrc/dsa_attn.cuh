@@ -41,6 +41,10 @@ struct AttnArgs {
     float* lse;                  //               [B, H_q]
     float* out_part;             // n_split > 1:  [B, H_q, n_split, D]
     float* lse_part;             //               [B, H_q, n_split]
+    // phase-2 selection with n_split > 1: per-split candidates, reduced by the combine kernel
+    float* sel_val_part;         // [B, H_q, n_split] lowest logit (base 2) among this split's candidates
+    int* sel_off_part;           // [B, H_q, n_split] its distance behind the query, -1 if none
+    int* sel_k;                  // [B, H_q] trace entry to write, -1 if this request selects nothing
 };
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, bool valid) {
@@ -115,7 +119,7 @@ __device__ __forceinline__ void group_sum_all(float (&x)[V], int lr) {
     for (int v = 0; v < V; ++v) x[v] = __shfl_sync(FULL, mine, v * (LPR / V), LPR);
 }
 
-template <typename T, int D, int G, int TILE_N, int STAGES, bool HEADMASK>
+template <typename T, int D, int G, int TILE_N, int STAGES, bool HEADMASK, bool SELECT = false>
 struct AttnCfg {
     static constexpr int VEC = Elem<T>::VEC;
     static constexpr int LPR = D / VEC;                 // lanes per row
@@ -125,33 +129,37 @@ struct AttnCfg {
     static constexpr int TILE_BYTES = TILE_N * ROW_BYTES;
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;  // K tile then V tile
     static constexpr int PIPE_BYTES = STAGES * STAGE_BYTES;
-    static constexpr int MERGE_BYTES = NG * G * (D + 2) * 4;
+    static constexpr int MSTRIDE = D + 4;               // merge record: acc[D], m, l, best logit, its position
+    static constexpr int MERGE_BYTES = NG * G * MSTRIDE * 4;
     static constexpr int SLOTS = HEADMASK ? G : 1;
     static_assert(LPR <= 32 && TILE_N % NG == 0 && R >= 1, "bad tiling");
     __host__ __device__ static constexpr int big_bytes() {
         return PIPE_BYTES > MERGE_BYTES ? PIPE_BYTES : MERGE_BYTES;
     }
-    // dynamic shared memory: [pipeline / merge area][row offsets int64 x chunk][head bits][bitmaps]
+    // dynamic shared memory:
+    // [pipeline / merge area][row offsets int64 x chunk][row positions int32 x chunk][head bits][bitmaps]
     __host__ static size_t smem_bytes(int chunk, int bitmap_words) {
         size_t b = big_bytes();
         b += (size_t)chunk * 8;
+        if (SELECT) b += (size_t)chunk * 4;
         if (HEADMASK) b += (size_t)((chunk + 15) / 16) * 16;
         b += (size_t)SLOTS * bitmap_words * 4;
         return b;
     }
 };
 
-template <typename T, int D, int G, int TILE_N, int STAGES, bool HEADMASK>
+template <typename T, int D, int G, int TILE_N, int STAGES, bool HEADMASK, bool SELECT>
 __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
-    using C = AttnCfg<T, D, G, TILE_N, STAGES, HEADMASK>;
-    constexpr int VEC = C::VEC, LPR = C::LPR, NG = C::NG, R = C::R, SLOTS = C::SLOTS;
+    using C = AttnCfg<T, D, G, TILE_N, STAGES, HEADMASK, SELECT>;
+    constexpr int VEC = C::VEC, LPR = C::LPR, NG = C::NG, R = C::R, SLOTS = C::SLOTS, MS = C::MSTRIDE;
     constexpr unsigned ALLBITS = (1u << SLOTS) - 1u;
 
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_warp[NT / 32];
     unsigned char* pipe = smem;
     int64_t* rowoff = reinterpret_cast<int64_t*>(smem + C::big_bytes());
-    unsigned char* hbits = reinterpret_cast<unsigned char*>(rowoff + a.chunk);
+    int* rowpos = reinterpret_cast<int*>(rowoff + a.chunk);
+    unsigned char* hbits = reinterpret_cast<unsigned char*>(rowpos + (SELECT ? a.chunk : 0));
     unsigned* bitmaps = reinterpret_cast<unsigned*>(hbits + (HEADMASK ? ((a.chunk + 15) / 16) * 16 : 0));
 
     const int tid = threadIdx.x;
@@ -167,11 +175,21 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     auto write_empty = [&]() {
         // nothing kept in this split: lse = -inf (and out = 0 when this block owns the result)
         if (a.n_split > 1) {
-            if (tid < G) a.lse_part[((int64_t)b * a.H_q + kvh * G + tid) * a.n_split + split] = -INFINITY;
+            if (tid < G) {
+                const int64_t row = (int64_t)b * a.H_q + kvh * G + tid;
+                a.lse_part[row * a.n_split + split] = -INFINITY;
+                if (SELECT) {
+                    a.sel_val_part[row * a.n_split + split] = INFINITY;
+                    a.sel_off_part[row * a.n_split + split] = -1;
+                    a.sel_k[row] = m.sel_k;
+                }
+            }
         } else {
             for (int i = tid; i < G * D; i += NT)
                 Elem<T>::store(a.out, ((int64_t)b * a.H_q + kvh * G) * D + i, 0.f);
             if (tid < G) a.lse[(int64_t)b * a.H_q + kvh * G + tid] = -INFINITY;
+            if (SELECT && tid < G && m.sel_k >= 0)
+                a.mask.skip_offsets[((int64_t)b * a.H_q + kvh * G + tid) * a.mask.trace_len + m.sel_k] = -1;
         }
     };
 
@@ -203,6 +221,7 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
                 off = (int64_t)b * a.stride_b + (int64_t)pos * a.stride_tok;
             }
             rowoff[slot] = off + head_off;
+            if (SELECT) rowpos[slot] = pos;
             if (HEADMASK) hbits[slot] = (unsigned char)bits;
         });
     const int n_rows = min(total - r0, a.chunk);
@@ -248,9 +267,14 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
             for (int e = 0; e < VEC; ++e) qf[g][e] *= a.scale_log2;
         }
     }
+    // selection: lowest logit among the attended decode keys that are not sinks, per head
+    float bestv[G];
+    int bestp[G];
+    const int cand_lo = m.L_p + a.mask.n_sink;
     float acc[G][VEC], mrun[G], lrun[G];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
+        bestv[g] = INFINITY; bestp[g] = 0x7fffffff;
         mrun[g] = -INFINITY; lrun[g] = 0.f;
 #pragma unroll
         for (int e = 0; e < VEC; ++e) acc[g][e] = 0.f;
@@ -299,10 +323,16 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
             const bool valid = r < n_rows;
             unsigned bits = ALLBITS;
             if (HEADMASK) bits = valid ? hbits[r] : 0u;
+            int pos = 0;
+            if (SELECT) pos = valid ? rowpos[r] : 0;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const bool on = valid && (!HEADMASK || ((bits >> g) & 1u));
                 if (!on) s[g * R + i] = -INFINITY;
+                // rows arrive in ascending position, so a strict "<" keeps the oldest of equal logits
+                if (SELECT && on && pos >= cand_lo && s[g * R + i] < bestv[g]) {
+                    bestv[g] = s[g * R + i]; bestp[g] = pos;
+                }
             }
         }
         // online softmax update, then s becomes the weights p
@@ -345,25 +375,28 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     __syncthreads();                          // pipeline memory is free: reuse it for the merge
 
     // ---- merge the lane groups ---------------------------------------------------------------
-    float* mg = reinterpret_cast<float*>(pipe);           // [NG][G][D + 2]: acc, then m, l
+    float* mg = reinterpret_cast<float*>(pipe);           // [NG][G][MS]: acc, m, l, best logit, its position
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        float* dst = mg + ((int64_t)gid * G + g) * (D + 2);
+        float* dst = mg + ((int64_t)gid * G + g) * MS;
 #pragma unroll
         for (int e = 0; e < VEC; ++e) dst[lr * VEC + e] = acc[g][e];
-        if (lr == 0) { dst[D] = mrun[g]; dst[D + 1] = lrun[g]; }
+        if (lr == 0) {
+            dst[D] = mrun[g]; dst[D + 1] = lrun[g];
+            if (SELECT) { dst[D + 2] = bestv[g]; dst[D + 3] = __int_as_float(bestp[g]); }
+        }
     }
     __syncthreads();
     for (int i = tid; i < G * D; i += NT) {
         const int g = i / D, d = i - g * D;
         float M = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < NG; ++j) M = fmaxf(M, mg[((int64_t)j * G + g) * (D + 2) + D]);
+        for (int j = 0; j < NG; ++j) M = fmaxf(M, mg[((int64_t)j * G + g) * MS + D]);
         float num = 0.f, den = 0.f;
         if (M != -INFINITY) {
 #pragma unroll
             for (int j = 0; j < NG; ++j) {
-                const float* src = mg + ((int64_t)j * G + g) * (D + 2);
+                const float* src = mg + ((int64_t)j * G + g) * MS;
                 const float w = fast_exp2(src[D] - M);
                 num = fmaf(w, src[d], num);
                 den = fmaf(w, src[D + 1], den);
@@ -372,20 +405,47 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
         const float o = den > 0.f ? num / den : 0.f;
         const float l = den > 0.f ? (M + log2f(den)) * LN2 : -INFINITY;
         const int h = kvh * G + g;
+        const int64_t row = (int64_t)b * a.H_q + h;
         if (a.n_split > 1) {
-            a.out_part[(((int64_t)b * a.H_q + h) * a.n_split + split) * D + d] = o;
-            if (d == 0) a.lse_part[((int64_t)b * a.H_q + h) * a.n_split + split] = l;
+            a.out_part[(row * a.n_split + split) * D + d] = o;
+            if (d == 0) a.lse_part[row * a.n_split + split] = l;
         } else {
-            Elem<T>::store(a.out, ((int64_t)b * a.H_q + h) * D + d, o);
-            if (d == 0) a.lse[(int64_t)b * a.H_q + h] = l;
+            Elem<T>::store(a.out, row * D + d, o);
+            if (d == 0) a.lse[row] = l;
+        }
+        if (SELECT && d == 0) {
+            // lowest logit over the lane groups; equal logits go to the oldest key
+            float bv = INFINITY;
+            int bp = 0x7fffffff;
+#pragma unroll
+            for (int j = 0; j < NG; ++j) {
+                const float* src = mg + ((int64_t)j * G + g) * MS;
+                const float v = src[D + 2];
+                const int pp = __float_as_int(src[D + 3]);
+                if (v < bv || (v == bv && pp < bp)) { bv = v; bp = pp; }
+            }
+            const int off = bp == 0x7fffffff ? -1 : (m.S - 1) - bp;
+            if (a.n_split > 1) {
+                a.sel_val_part[row * a.n_split + split] = bv;
+                a.sel_off_part[row * a.n_split + split] = off;
+                a.sel_k[row] = m.sel_k;
+            } else if (m.sel_k >= 0) {
+                a.mask.skip_offsets[row * a.mask.trace_len + m.sel_k] = off;
+            }
         }
     }
 }
 
 // ---- split combine: one block per (request, query head), one thread per output element -------
+// With sel_k != nullptr it also finishes Algorithm 1's selection: the lowest candidate logit over
+// the splits (equal logits: the oldest key, i.e. the largest distance) becomes trace entry sel_k.
 template <typename T>
 __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const float* __restrict__ lse_part,
-                                   int D, int n_split, void* out, float* lse) {
+                                   int D, int n_split, void* out, float* lse,
+                                   const float* __restrict__ sel_val_part = nullptr,
+                                   const int* __restrict__ sel_off_part = nullptr,
+                                   const int* __restrict__ sel_k = nullptr, int* trace = nullptr,
+                                   int trace_len = 0) {
     const int64_t row = blockIdx.x;
     const float* lp = lse_part + row * n_split;
     float M = -INFINITY;
@@ -406,6 +466,19 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
         Elem<T>::store(out, row * D + d, num * inv);
     }
     if (threadIdx.x == 0 && lse) lse[row] = den > 0.f ? M + logf(den) : -INFINITY;
+    if (threadIdx.x == 0 && sel_k != nullptr) {
+        const int k = sel_k[row];
+        if (k >= 0) {
+            float bv = INFINITY;
+            int bo = -1;
+            for (int i = 0; i < n_split; ++i) {
+                const float v = sel_val_part[row * n_split + i];
+                const int o = sel_off_part[row * n_split + i];
+                if (o >= 0 && (v < bv || (v == bv && o > bo))) { bv = v; bo = o; }
+            }
+            trace[row * trace_len + k] = bo;
+        }
+    }
 }
 
 // ---- debug export of the kept positions: one block per (request, mask head) ------------------

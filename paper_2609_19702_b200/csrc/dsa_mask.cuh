@@ -23,7 +23,8 @@ struct MaskArgs {
     int n_att;                 // N_att
     int stride;                // grid_w + row_extra (GRID)
     int n_sink;                // first decode tokens that are always kept (attention sinks)
-    const int* skip_offsets;   // [B, mask_heads, trace_len] (LIST)
+    int select;                // LIST: also run Algorithm 1's phase-2 selection and extend the trace
+    int* skip_offsets;         // [B, mask_heads, trace_len] (LIST); written when select is set
     int mask_heads;
     int trace_len;
     int bitmap_words;          // 32-bit words per LIST bitmap = ceil(window / 32)
@@ -40,6 +41,7 @@ struct ReqMask {
     int prefix;   // positions [0, prefix) are always kept: the prompt and the sinks older than the window
     int sink_end; // positions below this are sinks or prompt (kept even where the mask skips them)
     int n_act;    // LIST: active skip entries
+    int sel_k;    // LIST with selection: trace entry this step appends (-1: no selection at this step)
     int dstar;    // GRID: column distance of the partly kept class (-1: keep none below T)
     int need;     // GRID: how many distances of class dstar are kept (lowest first)
     bool keep_all;// nothing skipped at this position
@@ -60,7 +62,7 @@ __device__ __forceinline__ ReqMask req_mask_setup(const MaskArgs& a, int seq_len
     m.S = max(0, min(seq_len, max_seq_len));
     m.L_p = max(0, min(prompt_len, m.S));
     m.p = m.S - m.L_p;
-    m.n_act = 0; m.dstar = -1; m.need = 0; m.keep_all = true;
+    m.n_act = 0; m.dstar = -1; m.need = 0; m.keep_all = true; m.sel_k = -1;
     m.prefix = m.L_p; m.sink_end = m.L_p;
     if (a.mode == MODE_DENSE) {
         m.T = m.p - 1; m.n_win = m.p; m.w_lo = m.L_p;
@@ -76,6 +78,8 @@ __device__ __forceinline__ ReqMask req_mask_setup(const MaskArgs& a, int seq_len
     if (a.mode == MODE_LIST) {
         m.n_act = min(min(t - (a.n_att - 1), a.window - a.n_att), a.trace_len);
         m.keep_all = m.n_act <= 0;
+        // phase 2 (t < N_r) with |skip_idx| < N_r - N_att: steps N_att-1 .. N_r-2 select entry t-(N_att-1)
+        if (a.select && t <= a.window - 2 && t - (a.n_att - 1) < a.trace_len) m.sel_k = t - (a.n_att - 1);
         return m;
     }
     // GRID: keep the N_att - 1 best of [0, T) under (column distance, distance), plus T itself.

@@ -62,3 +62,22 @@ def attention(q: Sequence[float], keys: Sequence[Sequence[float]], values: Seque
     d = len(values[0])
     out = [math.fsum(w[j] * values[j][i] for j in range(len(values))) for i in range(d)]
     return out, lse
+
+
+def argmin_trace(q_steps: Sequence[Sequence[float]], keys: Sequence[Sequence[float]], n_r: int, n_att: int,
+                 scale: float, n_sink: int = 0) -> List[int]:
+    """Algorithm 1's own selection simulated in distance space: at steps N_att-1 .. N_r-2 the
+    attended decode key (sinks excluded) with the lowest logit is skipped from then on; equal
+    logits go to the lowest key index.  Returns the distances in selection order."""
+    skipped: List[int] = []
+    for s in range(n_att - 1, n_r - 1):
+        best = None
+        for o in range(s, -1, -1):                     # oldest key first, strict "<" keeps it on ties
+            j = s - o
+            if o in skipped or j < n_sink:
+                continue
+            logit = scale * math.fsum(a * b for a, b in zip(q_steps[s], keys[j]))
+            if best is None or logit < best[0]:
+                best = (logit, o)
+        skipped.append(best[1])
+    return skipped

@@ -312,6 +312,32 @@ def test_select_argmin_over_decode_keys_only():
     assert j2 == 0                               # ties: lowest cache index
 
 
+def test_replay_with_argmin_selection_against_distance_space_simulation():
+    rng = np.random.default_rng(21)
+    for n_r, n_att, n_sink, d in ((12, 4, 0, 8), (20, 7, 2, 5), (9, 2, 1, 16), (16, 15, 0, 4)):
+        steps = 2 * n_r + 3
+        q = rng.standard_normal((steps, d))
+        k = rng.standard_normal((steps, d))
+        want = brute.argmin_trace(q.tolist(), k.tolist(), n_r, n_att, 0.4, n_sink)
+        for t in (0, n_att - 1, n_att, n_r - 2, n_r - 1, steps - 1):
+            idx, tr = ora.replay_argmin(t, n_r, n_att, q, d, k.reshape(-1), np.arange(steps) * d, d, 0.4, n_sink)
+            n_sel = min(max(t - (n_att - 1) + 1, 0), n_r - n_att)
+            assert tr.tolist() == want[:n_sel]
+            # the same trace fed back as an input reproduces the attended set
+            idx2, _ = ora.replay(t, n_r, n_att, ora.SEL_TRACE, want)
+            assert idx.tolist() == idx2.tolist()
+    # the selected key really carries the lowest softmax weight among the attended decode keys
+    n_r, n_att, d = 10, 4, 6
+    q = rng.standard_normal((30, d))
+    k = rng.standard_normal((30, d))
+    _, tr = ora.replay_argmin(29, n_r, n_att, q, d, k.reshape(-1), np.arange(30) * d, d, 1.0)
+    for i, o in enumerate(tr.tolist()):
+        s_step = n_att - 1 + i
+        idx, _ = ora.replay(s_step, n_r, n_att, ora.SEL_TRACE, tr.tolist())
+        w = torch.softmax(torch.from_numpy(k[idx] @ q[s_step]), 0)
+        assert int(idx[int(torch.argmin(w))]) == s_step - o
+
+
 # ---------------------------------------------------------------- the batched driver
 
 def _brute_decode(inp, kept_fn):
