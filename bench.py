@@ -250,6 +250,84 @@ def per_config_table(torch, dsa, synth, dev, peak):
     return rows
 
 
+def decode_loop_bench(torch, dsa, synth, dev):
+    """Whole-image decode loop (one layer's attention): 1024 image tokens after a 50-token prompt,
+    batch 16, 32/32 heads, head_dim 128 -- the shape of the paper's Lumina-mGPT latency runs.
+    Every step appends the new token's K/V and attends; the step is captured once as a CUDA
+    graph and replayed.  Sparse: bounded ring cache, window 512, N_att 52 (95 % sparsity), grid
+    mask.  Dense: full linear cache."""
+    b, h, d, l_p, grid = 16, 32, 128, 50, 32
+    steps = grid * grid
+    s_max = l_p + steps
+    row = h * d
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(synth.BASE_SEED + 77)
+    res = {"batch": b, "heads": h, "head_dim": d, "prompt_len": l_p, "image_tokens": steps}
+    for mode in ("dense", "sparse"):
+        ring = 512 if mode == "sparse" else 0
+        cap = l_p + ring if ring else s_max
+        kc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        vc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        q = torch.randn((b, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        k_new, v_new = q.clone(), q.clone()
+        seq = torch.full((b,), l_p, dtype=torch.int32, device=dev)
+        pl = torch.full((b,), l_p, dtype=torch.int32, device=dev)
+        prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d),
+                           seq_len=seq, prompt_len=pl, num_kv_heads=h, max_seq_len=s_max, max_prompt_len=l_p,
+                           ring_size=ring)
+        diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 52, grid, 0) if mode == "sparse" else None
+        out, lse = dsa.alloc_outputs(prob)
+        ws = dsa.alloc_workspace(prob, diag)
+
+        def step():
+            dsa.dsa_append_kv(prob, k_new, v_new, advance=True)
+            if diag is None:
+                dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+            else:
+                dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+
+        step()                                             # eager warm-up (one-time kernel set-up)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        best = None
+        for _ in range(3):
+            seq.fill_(l_p)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        assert int(seq[0].item()) == s_max
+        # the last step alone (the paper's per-step breakdown is taken there)
+        seq.fill_(s_max - 1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        e0.record()
+        for _ in range(reps):
+            seq.fill_(s_max - 1)
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        plan = dsa.dsa_query_plan(prob, diag)
+        res[mode] = {"ms_per_image": round(best, 3), "us_per_step_mean": round(best / steps * 1e3, 2),
+                     "us_last_step": round(e0.elapsed_time(e1) / reps * 1e3, 2),
+                     "cache_GB": round(2 * kc.numel() * 2 / 1e9, 3), "n_split": plan.n_split,
+                     "launches_per_step": plan.launches + 2}
+        del kc, vc, graph
+        torch.cuda.empty_cache()
+    res["speedup_per_image"] = round(res["dense"]["ms_per_image"] / res["sparse"]["ms_per_image"], 3)
+    res["speedup_last_step"] = round(res["dense"]["us_last_step"] / res["sparse"]["us_last_step"], 3)
+    res["cache_ratio"] = round(res["dense"]["cache_GB"] / res["sparse"]["cache_GB"], 3)
+    return res
+
+
 def run_ours(args):
     import torch
     from paper_2609_19702_b200 import build as cuda_build
@@ -389,11 +467,12 @@ def run_ours(args):
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
-    per_config = None
+    per_config = decode_loop = None
     if args.all_configs and rank == 0 and world == 1:
         del inputs, prob, out, lse
         torch.cuda.empty_cache()
         per_config = per_config_table(torch, dsa, synth, dev, peak)
+        decode_loop = decode_loop_bench(torch, dsa, synth, dev)
 
     if rank == 0:
         line = {
@@ -413,6 +492,7 @@ def run_ours(args):
         }
         if per_config is not None:
             line["per_config"] = per_config
+            line["decode_loop"] = decode_loop
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -100,6 +100,17 @@ typedef struct dsa_problem {
                                /* call then plans for max_seq_len kept tokens)                     */
     int32_t split_tokens;      /* kept tokens handled by one thread block; 0 = library chooses.    */
                                /* Rounded up to the tile size, at most 1024                        */
+    /* Bounded cache (Algorithm 1, phase 3: "evict oldest KV"; footprint N_r + L_p of Section 4's
+     * cost analysis).  ring_size == 0: every token is stored at its logical position.
+     * ring_size > 0: the prompt and the first ring_sinks decode tokens are stored at their logical
+     * positions; decode token j >= ring_sinks is stored at position
+     * L_p + ring_sinks + (j - ring_sinks) mod ring_size, overwriting the token that left the
+     * window ring_size steps earlier.  seq_len stays the LOGICAL length.  Needs
+     * max_prompt_len > 0; sparse calls need window <= ring_size and n_sink <= ring_sinks; the
+     * dense call is refused.  The cache then needs max_prompt_len + ring_sinks + ring_size
+     * tokens per request instead of max_seq_len. */
+    int32_t ring_size;
+    int32_t ring_sinks;
 } dsa_problem;
 
 /*
@@ -209,8 +220,21 @@ DSA_API int32_t dsa_combine_splits(const float *out_part, const float *lse_part,
                            void *out, float *lse, int32_t out_dtype, void *stream);
 
 /*
+ * Append the K/V rows of the token being decoded (the cache write that precedes attention in a
+ * decode step; with a bounded cache this is also Algorithm 1's eviction, since the new token
+ * takes the slot of the one that left the window).  k_new, v_new: device [B, H_kv, D] in
+ * problem->dtype.  The rows of request b go to logical position seq_len[b] (the value BEFORE
+ * the call); a request whose seq_len is already max_seq_len is left alone.  With advance != 0
+ * seq_len[b] is then incremented on the device (two launches), so that a captured sequence
+ * "append, attend" can be replayed step after step without the host touching seq_len.
+ */
+DSA_API int32_t dsa_append_kv(const dsa_problem *problem, const void *k_new, const void *v_new,
+                              int32_t advance, void *stream);
+
+/*
  * The kept cache positions, produced by the same device code that the sparse attention kernel
  * uses to decide which rows to read (Algorithm 1: K_p, then window - skip_idx as positions).
+ * Positions are LOGICAL (before any ring mapping).
  * idx_out [B, mask_heads, max_kept] int32, ascending, entries beyond the count untouched;
  * count_out [B, mask_heads] int32 holds the full count even when it exceeds max_kept.
  * mask_heads is diag->mask_heads for LIST and 1 otherwise; diag == NULL reports the dense set.

@@ -23,7 +23,7 @@ DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
 EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_workspace_size",
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
            "dsa_combine_splits", "dsa_debug_kept_indices",
-           "dsa_decode_attention_static_scratch"]
+           "dsa_decode_attention_static_scratch", "dsa_append_kv"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -37,7 +37,8 @@ class dsa_problem(ctypes.Structure):
                 ("block_table", ctypes.c_void_p),
                 ("max_blocks", ctypes.c_int32), ("block_size", ctypes.c_int32),
                 ("num_blocks", ctypes.c_int32), ("max_seq_len", ctypes.c_int32),
-                ("max_prompt_len", ctypes.c_int32), ("split_tokens", ctypes.c_int32)]
+                ("max_prompt_len", ctypes.c_int32), ("split_tokens", ctypes.c_int32),
+                ("ring_size", ctypes.c_int32), ("ring_sinks", ctypes.c_int32)]
 
 
 class dsa_diag_params(ctypes.Structure):
@@ -77,6 +78,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_combine_splits.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp]
     lib.dsa_decode_attention_static_scratch.restype = i32
     lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
+    lib.dsa_append_kv.restype = i32
+    lib.dsa_append_kv.argtypes = [vp, vp, vp, i32, vp]
     lib.dsa_debug_kept_indices.restype = i32
     lib.dsa_debug_kept_indices.argtypes = [vp, vp, vp, vp, i32, vp]
     return lib
@@ -134,6 +137,8 @@ class Problem:
     num_blocks: int = 0
     sm_scale: float = 0.0
     split_tokens: int = 0
+    ring_size: int = 0                    # > 0: bounded cache, decode tokens live in a ring
+    ring_sinks: int = 0
 
     def c_struct(self) -> dsa_problem:
         b, hq, d = self.q.shape
@@ -155,6 +160,7 @@ class Problem:
         p.max_seq_len = int(self.max_seq_len)
         p.max_prompt_len = int(self.max_prompt_len)
         p.split_tokens = int(self.split_tokens)
+        p.ring_size, p.ring_sinks = int(self.ring_size), int(self.ring_sinks)
         return p
 
 
@@ -265,6 +271,16 @@ def dsa_combine_splits(out_part: torch.Tensor, lse_part: torch.Tensor, out: torc
     _check("dsa_combine_splits",
            _lib.dsa_combine_splits(_dptr(out_part), _dptr(lse_part), b, hq, d, n_split, _dptr(out),
                                    _dptr(lse), _dtype_code(out), _stream(stream)))
+
+
+def dsa_append_kv(problem: Problem, k_new: torch.Tensor, v_new: torch.Tensor, advance: bool = False,
+                  stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Write the new token's K/V rows [B, H_kv, D] at logical position seq_len[b]; optionally
+    increment seq_len on the device afterwards."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.dtype == problem.q.dtype
+    p = problem.c_struct()
+    _check("dsa_append_kv", _lib.dsa_append_kv(_ref(p), _dptr(k_new), _dptr(v_new), 1 if advance else 0,
+                                               _stream(stream)))
 
 
 def dsa_debug_kept_indices(problem: Problem, diag: Optional[Diag], max_kept: int,

@@ -101,6 +101,13 @@ int32_t dispatch(int dtype, int D, int G, bool hm, bool sel, F&& f) {
     return DSA_ERR_UNSUPPORTED;
 }
 
+// Tokens one request can hold: its logical maximum, or prompt + sinks + ring when bounded.
+int64_t physical_capacity(const dsa_problem* p) {
+    if (p->ring_size > 0)
+        return std::min<int64_t>(p->max_seq_len, (int64_t)p->max_prompt_len + p->ring_sinks + p->ring_size);
+    return p->max_seq_len;
+}
+
 int32_t check_problem(const dsa_problem* p) {
     if (!p) return DSA_ERR_INVALID_ARG;
     if (p->batch < 0 || p->num_q_heads < 1 || p->num_kv_heads < 1) return DSA_ERR_INVALID_ARG;
@@ -117,9 +124,11 @@ int32_t check_problem(const dsa_problem* p) {
     const int64_t vec = p->dtype == DSA_BF16 ? 8 : 4;          // elements per 16 bytes
     if (p->stride_batch < 0 || p->stride_token < p->head_dim || p->stride_head < 0) return DSA_ERR_INVALID_ARG;
     if (p->stride_batch % vec || p->stride_token % vec || p->stride_head % vec) return DSA_ERR_INVALID_ARG;
+    if (p->ring_size < 0 || p->ring_sinks < 0) return DSA_ERR_INVALID_ARG;
+    if (p->ring_size > 0 && p->max_prompt_len < 1) return DSA_ERR_INVALID_ARG;   // capacity needs the bound
     if (p->block_table) {
         if (p->block_size < 1 || p->max_blocks < 1 || p->num_blocks < 1) return DSA_ERR_INVALID_ARG;
-        if ((int64_t)p->max_blocks * p->block_size < p->max_seq_len) return DSA_ERR_INVALID_ARG;
+        if ((int64_t)p->max_blocks * p->block_size < physical_capacity(p)) return DSA_ERR_INVALID_ARG;
     }
     return DSA_OK;
 }
@@ -129,6 +138,8 @@ int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
     if (d->mode != DSA_MASK_WINDOW && d->mode != DSA_MASK_GRID && d->mode != DSA_MASK_LIST)
         return DSA_ERR_INVALID_ARG;
     if (d->window < 1 || d->n_sink < 0) return DSA_ERR_INVALID_ARG;
+    // a bounded cache holds the last ring_size decode tokens and the first ring_sinks: nothing else can be kept
+    if (p->ring_size > 0 && (d->window > p->ring_size || d->n_sink > p->ring_sinks)) return DSA_ERR_INVALID_ARG;
     if (d->mode == DSA_MASK_WINDOW) return DSA_OK;
     if (d->n_att < 1 || d->n_att > d->window) return DSA_ERR_INVALID_ARG;
     if (d->mode == DSA_MASK_GRID) {
@@ -152,6 +163,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     if (rc != DSA_OK) return rc;
     rc = check_diag(p, d);
     if (rc != DSA_OK) return rc;
+    if (!d && p->ring_size > 0) return DSA_ERR_INVALID_ARG;    // dense attention needs every token
     const int G = p->num_q_heads / p->num_kv_heads;
     pl->G = G;
     pl->mode = !d ? MODE_DENSE
@@ -229,6 +241,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->block_table = p->block_table;
     a->max_blocks = p->max_blocks; a->block_size = p->block_size; a->num_blocks = p->num_blocks;
     a->max_seq_len = p->max_seq_len;
+    a->ring_size = p->ring_size; a->ring_sinks = p->ring_sinks;
     a->B = p->batch; a->H_q = p->num_q_heads; a->H_kv = p->num_kv_heads;
     const float scale = p->sm_scale > 0.f ? p->sm_scale : 1.f / sqrtf((float)p->head_dim);
     a->scale_log2 = scale * LOG2E;
@@ -366,6 +379,38 @@ int32_t dsa_combine_splits(const float* out_part, const float* lse_part, int32_t
     if (!out_part || !lse_part || !out) return DSA_ERR_INVALID_ARG;
     return launch_combine(out_part, lse_part, (int64_t)batch * num_q_heads, head_dim, n_split, out, lse,
                           out_dtype, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int32_t dsa_append_kv(const dsa_problem* problem, const void* k_new, const void* v_new, int32_t advance,
+                      void* stream) {
+    const int32_t rc = check_problem(problem);
+    if (rc != DSA_OK) return rc;
+    if (problem->batch == 0) return DSA_OK;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return DSA_ERR_INVALID_ARG;
+    Plan pl = {};
+    pl.mode = MODE_WINDOW;
+    pl.chunk = 0; pl.n_split = 1;
+    AttnArgs a;
+    fill_args(problem, nullptr, pl, &a);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const unsigned grid = (unsigned)(problem->batch * problem->num_kv_heads);
+    const int cap = problem->max_seq_len;
+    if (problem->dtype == DSA_BF16)
+        dsa_append_kv_kernel<__nv_bfloat16><<<grid, 32, 0, st>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_new),
+                                                              reinterpret_cast<const __nv_bfloat16*>(v_new),
+                                                              problem->head_dim, cap);
+    else
+        dsa_append_kv_kernel<float><<<grid, 32, 0, st>>>(a, reinterpret_cast<const float*>(k_new),
+                                                       reinterpret_cast<const float*>(v_new), problem->head_dim, cap);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (advance) {
+        dsa_advance_kernel<<<(problem->batch + 127) / 128, 128, 0, st>>>(const_cast<int*>(problem->seq_len),
+                                                                       problem->batch, cap);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return DSA_OK;
 }
 
 int32_t dsa_debug_kept_indices(const dsa_problem* problem, const dsa_diag_params* diag, int32_t* idx_out,

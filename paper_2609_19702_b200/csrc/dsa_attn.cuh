@@ -32,6 +32,7 @@ struct AttnArgs {
     const int* block_table;
     int max_blocks, block_size, num_blocks;
     int max_seq_len;
+    int ring_size, ring_sinks;   // bounded cache: decode tokens beyond the first ring_sinks live in a ring
     int B, H_q, H_kv;
     float scale_log2;            // sm_scale * log2(e)
     MaskArgs mask;
@@ -46,6 +47,24 @@ struct AttnArgs {
     int* sel_off_part;           // [B, H_q, n_split] its distance behind the query, -1 if none
     int* sel_k;                  // [B, H_q] trace entry to write, -1 if this request selects nothing
 };
+
+// Where token `pos` (logical cache position) of request b lives, as an element offset of its kv
+// head 0.  With a bounded cache (ring_size > 0) the prompt and the first ring_sinks decode tokens
+// are stored in order and every later decode token j sits in ring slot (j - ring_sinks) mod
+// ring_size behind them: the slot of the token it evicted ring_size steps earlier.
+__device__ __forceinline__ int64_t token_offset(const AttnArgs& a, int b, int L_p, int pos) {
+    if (a.ring_size > 0) {
+        const int first = L_p + a.ring_sinks;
+        if (pos >= first) pos = first + (pos - first) % a.ring_size;
+    }
+    if (a.block_table) {
+        const int bi = pos / a.block_size;
+        int blk = a.block_table[(int64_t)b * a.max_blocks + min(bi, a.max_blocks - 1)];
+        blk = max(0, min(blk, a.num_blocks - 1));
+        return (int64_t)blk * a.stride_b + (int64_t)(pos - bi * a.block_size) * a.stride_tok;
+    }
+    return (int64_t)b * a.stride_b + (int64_t)pos * a.stride_tok;
+}
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, bool valid) {
     const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -211,16 +230,7 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     const int64_t head_off = (int64_t)kvh * a.stride_head;
     const int total = enumerate_kept<NT, SLOTS>(a.mask, m, bitmaps, r0, r1, s_warp,
         [&](int slot, int pos, unsigned bits) {
-            int64_t off;
-            if (a.block_table) {
-                const int bi = pos / a.block_size;
-                int blk = a.block_table[(int64_t)b * a.max_blocks + bi];
-                blk = max(0, min(blk, a.num_blocks - 1));
-                off = (int64_t)blk * a.stride_b + (int64_t)(pos - bi * a.block_size) * a.stride_tok;
-            } else {
-                off = (int64_t)b * a.stride_b + (int64_t)pos * a.stride_tok;
-            }
-            rowoff[slot] = off + head_off;
+            rowoff[slot] = token_offset(a, b, m.L_p, pos) + head_off;
             if (SELECT) rowpos[slot] = pos;
             if (HEADMASK) hbits[slot] = (unsigned char)bits;
         });
@@ -479,6 +489,31 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
             trace[row * trace_len + k] = bo;
         }
     }
+}
+
+// ---- K/V append: the new token of every request goes to logical position seq_len[b] --------------
+// One block per (request, kv head); 16-byte copies.  k_new / v_new are [B, H_kv, D].
+template <typename T>
+__global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_new, const T* __restrict__ v_new,
+                                     int D, int capacity) {
+    const int kvh = blockIdx.x % a.H_kv, b = blockIdx.x / a.H_kv;
+    const int S = a.seq_len[b];
+    if (S < 0 || S >= capacity) return;                   // no room: the token is dropped
+    const int L_p = max(0, min(a.prompt_len[b], S));
+    const int64_t dst = token_offset(a, b, L_p, S) + (int64_t)kvh * a.stride_head;
+    const int64_t src = ((int64_t)b * a.H_kv + kvh) * D;
+    constexpr int VEC = 16 / (int)sizeof(T);
+    T* kc = reinterpret_cast<T*>(const_cast<void*>(a.k));
+    T* vc = reinterpret_cast<T*>(const_cast<void*>(a.v));
+    for (int i = threadIdx.x * VEC; i < D; i += blockDim.x * VEC) {
+        *reinterpret_cast<uint4*>(kc + dst + i) = *reinterpret_cast<const uint4*>(k_new + src + i);
+        *reinterpret_cast<uint4*>(vc + dst + i) = *reinterpret_cast<const uint4*>(v_new + src + i);
+    }
+}
+
+__global__ void dsa_advance_kernel(int* seq_len, int B, int capacity) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B && seq_len[b] >= 0 && seq_len[b] < capacity) seq_len[b] += 1;
 }
 
 // ---- debug export of the kept positions: one block per (request, mask head) ------------------
