@@ -250,41 +250,49 @@ def per_config_table(torch, dsa, synth, dev, peak):
     return rows
 
 
-def decode_loop_bench(torch, dsa, synth, dev):
-    """Whole-image decode loop (one layer's attention): 1024 image tokens after a 50-token prompt,
-    batch 16, 32/32 heads, head_dim 128 -- the shape of the paper's Lumina-mGPT latency runs.
-    Every step appends the new token's K/V and attends; the step is captured once as a CUDA
-    graph and replayed.  Sparse: bounded ring cache, window 512, N_att 52 (95 % sparsity), grid
-    mask.  Dense: full linear cache."""
+def decode_loop_bench(torch, dsa, synth, dev, n_layers=8):
+    """Whole-image decode loop: 1024 image tokens after a 50-token prompt, batch 16, 32/32 heads,
+    head_dim 128 -- the shape of the paper's Lumina-mGPT latency runs -- over `n_layers` layers,
+    each with its own KV cache (together larger than the L2).  Every step appends the new token's
+    K/V and attends, layer after layer; the step is captured once as a CUDA graph and replayed
+    1024 times.  Sparse: bounded ring cache, window 512, N_att 52 (95 % sparsity), grid mask.
+    Dense: full linear cache."""
     b, h, d, l_p, grid = 16, 32, 128, 50, 32
     steps = grid * grid
     s_max = l_p + steps
     row = h * d
     gen = torch.Generator(device=dev)
     gen.manual_seed(synth.BASE_SEED + 77)
-    res = {"batch": b, "heads": h, "head_dim": d, "prompt_len": l_p, "image_tokens": steps}
+    res = {"batch": b, "heads": h, "head_dim": d, "prompt_len": l_p, "image_tokens": steps, "layers": n_layers}
     for mode in ("dense", "sparse"):
         ring = 512 if mode == "sparse" else 0
         cap = l_p + ring if ring else s_max
-        kc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
-        vc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 52, grid, 0) if mode == "sparse" else None
         q = torch.randn((b, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         k_new, v_new = q.clone(), q.clone()
-        seq = torch.full((b,), l_p, dtype=torch.int32, device=dev)
-        pl = torch.full((b,), l_p, dtype=torch.int32, device=dev)
-        prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d),
-                           seq_len=seq, prompt_len=pl, num_kv_heads=h, max_seq_len=s_max, max_prompt_len=l_p,
-                           ring_size=ring)
-        diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 52, grid, 0) if mode == "sparse" else None
-        out, lse = dsa.alloc_outputs(prob)
-        ws = dsa.alloc_workspace(prob, diag)
+        layers = []
+        for _ in range(n_layers):
+            kc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+            vc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+            seq = torch.full((b,), l_p, dtype=torch.int32, device=dev)
+            pl = torch.full((b,), l_p, dtype=torch.int32, device=dev)
+            prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d),
+                               seq_len=seq, prompt_len=pl, num_kv_heads=h, max_seq_len=s_max,
+                               max_prompt_len=l_p, ring_size=ring)
+            out, lse = dsa.alloc_outputs(prob)
+            layers.append((prob, out, lse, dsa.alloc_workspace(prob, diag)))
 
         def step():
-            dsa.dsa_append_kv(prob, k_new, v_new, advance=True)
-            if diag is None:
-                dsa.dsa_decode_attention_dense(prob, out, lse, ws)
-            else:
-                dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+            for prob, out, lse, ws in layers:
+                dsa.dsa_append_kv(prob, k_new, v_new, advance=True)
+                if diag is None:
+                    dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+                else:
+                    dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+
+        def reset(value):
+            for prob, _, _, _ in layers:
+                prob.seq_len.fill_(value)
 
         step()                                             # eager warm-up (one-time kernel set-up)
         torch.cuda.synchronize()
@@ -293,7 +301,7 @@ def decode_loop_bench(torch, dsa, synth, dev):
             step()
         best = None
         for _ in range(3):
-            seq.fill_(l_p)
+            reset(l_p)
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
@@ -303,28 +311,29 @@ def decode_loop_bench(torch, dsa, synth, dev):
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1)
             best = ms if best is None else min(best, ms)
-        assert int(seq[0].item()) == s_max
+        assert int(layers[0][0].seq_len[0].item()) == s_max
         # the last step alone (the paper's per-step breakdown is taken there)
-        seq.fill_(s_max - 1)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 20
-        e0.record()
+        reps, last = 20, 0.0
         for _ in range(reps):
-            seq.fill_(s_max - 1)
+            reset(s_max - 1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
             graph.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        plan = dsa.dsa_query_plan(prob, diag)
-        res[mode] = {"ms_per_image": round(best, 3), "us_per_step_mean": round(best / steps * 1e3, 2),
-                     "us_last_step": round(e0.elapsed_time(e1) / reps * 1e3, 2),
-                     "cache_GB": round(2 * kc.numel() * 2 / 1e9, 3), "n_split": plan.n_split,
-                     "launches_per_step": plan.launches + 2}
-        del kc, vc, graph
+            e1.record()
+            torch.cuda.synchronize()
+            last += e0.elapsed_time(e1)
+        plan = dsa.dsa_query_plan(layers[0][0], diag)
+        cache_gb = n_layers * 2 * b * cap * row * 2 / 1e9
+        res[mode] = {"ms_per_image": round(best, 3), "us_per_step": round(best / steps * 1e3, 2),
+                     "us_per_layer_step": round(best / steps / n_layers * 1e3, 2),
+                     "us_last_step": round(last / reps * 1e3, 2), "cache_GB": round(cache_gb, 3),
+                     "n_split": plan.n_split, "launches_per_layer_step": plan.launches + 1}
+        del layers, graph
         torch.cuda.empty_cache()
     res["speedup_per_image"] = round(res["dense"]["ms_per_image"] / res["sparse"]["ms_per_image"], 3)
     res["speedup_last_step"] = round(res["dense"]["us_last_step"] / res["sparse"]["us_last_step"], 3)
     res["cache_ratio"] = round(res["dense"]["cache_GB"] / res["sparse"]["cache_GB"], 3)
+    res["ideal_last_step_byte_ratio"] = round((l_p + steps) / (l_p + 52), 3)
     return res
 
 

@@ -225,7 +225,7 @@ DSA_API int32_t dsa_combine_splits(const float *out_part, const float *lse_part,
  * takes the slot of the one that left the window).  k_new, v_new: device [B, H_kv, D] in
  * problem->dtype.  The rows of request b go to logical position seq_len[b] (the value BEFORE
  * the call); a request whose seq_len is already max_seq_len is left alone.  With advance != 0
- * seq_len[b] is then incremented on the device (two launches), so that a captured sequence
+ * seq_len[b] is then incremented on the device by the same kernel, so that a captured sequence
  * "append, attend" can be replayed step after step without the host touching seq_len.
  */
 DSA_API int32_t dsa_append_kv(const dsa_problem *problem, const void *k_new, const void *v_new,

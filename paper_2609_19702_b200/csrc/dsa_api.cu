@@ -196,15 +196,16 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     if (p->split_tokens > 0) {
         chunk = std::min(MAX_CHUNK, round_up(p->split_tokens, pl->tile));
     } else {
-        // Few (request, kv head) pairs: split until about two waves of blocks exist, but keep
-        // at least a few tiles per block.  Many pairs: as few splits as the row list allows.
+        // One block streams about 12 GB/s on its own, and a split costs the combine launch, so:
+        // split only while fewer than ~4 blocks per SM exist, never below 128 rows per block, and
+        // balance the splits (equal chunks rather than full ones plus a short tail).
         const int64_t pairs = (int64_t)std::max(p->batch, 1) * p->num_kv_heads;
-        const int64_t target = 2 * 8 * kNumSMs;
-        int64_t want_split = (target + pairs - 1) / pairs;
-        if (want_split < 1) want_split = 1;
-        int64_t c = (bound + want_split - 1) / want_split;
-        c = std::max<int64_t>(c, 64);
-        chunk = (int)std::min<int64_t>(MAX_CHUNK, round_up((int)std::min<int64_t>(c, MAX_CHUNK), pl->tile));
+        const int64_t target = 4 * kNumSMs;
+        int64_t want_split = std::max<int64_t>(1, (target + pairs - 1) / pairs);
+        want_split = std::min<int64_t>(want_split, std::max<int64_t>(1, bound / 128));
+        want_split = std::max<int64_t>(want_split, (bound + MAX_CHUNK - 1) / MAX_CHUNK);
+        const int64_t c = (bound + want_split - 1) / want_split;
+        chunk = std::min(MAX_CHUNK, round_up((int)c, pl->tile));
     }
     pl->chunk = chunk;
     pl->n_split = (int)((bound + chunk - 1) / chunk);
@@ -238,6 +239,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->q = p->q; a->k = p->k_cache; a->v = p->v_cache;
     a->stride_b = p->stride_batch; a->stride_tok = p->stride_token; a->stride_head = p->stride_head;
     a->seq_len = p->seq_len; a->prompt_len = p->prompt_len;
+    a->seq_len_rw = const_cast<int*>(p->seq_len);
     a->block_table = p->block_table;
     a->max_blocks = p->max_blocks; a->block_size = p->block_size; a->num_blocks = p->num_blocks;
     a->max_seq_len = p->max_seq_len;
@@ -393,24 +395,18 @@ int32_t dsa_append_kv(const dsa_problem* problem, const void* k_new, const void*
     AttnArgs a;
     fill_args(problem, nullptr, pl, &a);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const unsigned grid = (unsigned)(problem->batch * problem->num_kv_heads);
+    const unsigned grid = (unsigned)problem->batch;
     const int cap = problem->max_seq_len;
     if (problem->dtype == DSA_BF16)
-        dsa_append_kv_kernel<__nv_bfloat16><<<grid, 32, 0, st>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_new),
-                                                              reinterpret_cast<const __nv_bfloat16*>(v_new),
-                                                              problem->head_dim, cap);
+        dsa_append_kv_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_new),
+                                                               reinterpret_cast<const __nv_bfloat16*>(v_new),
+                                                               problem->head_dim, cap, advance != 0);
     else
-        dsa_append_kv_kernel<float><<<grid, 32, 0, st>>>(a, reinterpret_cast<const float*>(k_new),
-                                                       reinterpret_cast<const float*>(v_new), problem->head_dim, cap);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(e);
-    if (advance) {
-        dsa_advance_kernel<<<(problem->batch + 127) / 128, 128, 0, st>>>(const_cast<int*>(problem->seq_len),
-                                                                       problem->batch, cap);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
-    return DSA_OK;
+        dsa_append_kv_kernel<float><<<grid, 256, 0, st>>>(a, reinterpret_cast<const float*>(k_new),
+                                                        reinterpret_cast<const float*>(v_new), problem->head_dim, cap,
+                                                        advance != 0);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
 int32_t dsa_debug_kept_indices(const dsa_problem* problem, const dsa_diag_params* diag, int32_t* idx_out,

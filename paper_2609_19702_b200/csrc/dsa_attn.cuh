@@ -28,6 +28,7 @@ struct AttnArgs {
     const void* v;
     int64_t stride_b, stride_tok, stride_head;
     const int* seq_len;
+    int* seq_len_rw;             // same array, for the append call that advances it
     const int* prompt_len;
     const int* block_table;
     int max_blocks, block_size, num_blocks;
@@ -492,28 +493,30 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
 }
 
 // ---- K/V append: the new token of every request goes to logical position seq_len[b] --------------
-// One block per (request, kv head); 16-byte copies.  k_new / v_new are [B, H_kv, D].
+// One block per request copies its H_kv rows of K and of V (16-byte pieces) and then, if asked,
+// advances seq_len[b]; no other block reads that entry, so the update needs no further ordering.
+// k_new / v_new are [B, H_kv, D].
 template <typename T>
 __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_new, const T* __restrict__ v_new,
-                                     int D, int capacity) {
-    const int kvh = blockIdx.x % a.H_kv, b = blockIdx.x / a.H_kv;
+                                     int D, int capacity, bool advance) {
+    const int b = blockIdx.x;
     const int S = a.seq_len[b];
     if (S < 0 || S >= capacity) return;                   // no room: the token is dropped
     const int L_p = max(0, min(a.prompt_len[b], S));
-    const int64_t dst = token_offset(a, b, L_p, S) + (int64_t)kvh * a.stride_head;
-    const int64_t src = ((int64_t)b * a.H_kv + kvh) * D;
+    const int64_t dst0 = token_offset(a, b, L_p, S);
     constexpr int VEC = 16 / (int)sizeof(T);
     T* kc = reinterpret_cast<T*>(const_cast<void*>(a.k));
     T* vc = reinterpret_cast<T*>(const_cast<void*>(a.v));
-    for (int i = threadIdx.x * VEC; i < D; i += blockDim.x * VEC) {
-        *reinterpret_cast<uint4*>(kc + dst + i) = *reinterpret_cast<const uint4*>(k_new + src + i);
-        *reinterpret_cast<uint4*>(vc + dst + i) = *reinterpret_cast<const uint4*>(v_new + src + i);
+    const int per_row = D / VEC;
+    for (int i = threadIdx.x; i < a.H_kv * per_row; i += blockDim.x) {
+        const int kvh = i / per_row, c = (i - kvh * per_row) * VEC;
+        const int64_t dst = dst0 + (int64_t)kvh * a.stride_head + c;
+        const int64_t src = ((int64_t)b * a.H_kv + kvh) * D + c;
+        *reinterpret_cast<uint4*>(kc + dst) = *reinterpret_cast<const uint4*>(k_new + src);
+        *reinterpret_cast<uint4*>(vc + dst) = *reinterpret_cast<const uint4*>(v_new + src);
     }
-}
-
-__global__ void dsa_advance_kernel(int* seq_len, int B, int capacity) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < B && seq_len[b] >= 0 && seq_len[b] < capacity) seq_len[b] += 1;
+    __syncthreads();                                       // every thread has read S
+    if (advance && threadIdx.x == 0) a.seq_len_rw[b] = S + 1;
 }
 
 // ---- debug export of the kept positions: one block per (request, mask head) ------------------
