@@ -13,12 +13,13 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdsa.so")
 SOURCES = ["dsa_api.cu"]
-HEADERS = ["dsa_attn.cuh", "dsa_mask.cuh", os.path.join("..", "..", "include", "dsa.h")]
+HEADERS = ["dsa_attn.cuh", "dsa_attn_persistent.cuh", "dsa_tile.cuh", "dsa_common.cuh", "dsa_mask.cuh",
+           os.path.join("..", "..", "include", "dsa.h")]
 
 
 def _newest_source_mtime() -> float:
     paths = [os.path.join(CSRC, s) for s in SOURCES + HEADERS]
-    return max(os.path.getmtime(p) for p in paths)
+    return max(os.path.getmtime(p) for p in paths if os.path.exists(p))
 
 
 def build(force: bool = False, verbose: bool = False, out: str = LIB) -> str:

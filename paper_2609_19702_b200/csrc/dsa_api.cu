@@ -236,6 +236,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
 }
 
 void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, AttnArgs* a) {
+    *a = AttnArgs{};
     a->q = p->q; a->k = p->k_cache; a->v = p->v_cache;
     a->stride_b = p->stride_batch; a->stride_tok = p->stride_token; a->stride_head = p->stride_head;
     a->seq_len = p->seq_len; a->prompt_len = p->prompt_len;
@@ -258,6 +259,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.trace_len = (d && pl.mode == MODE_LIST) ? d->trace_len : 0;
     a->mask.bitmap_words = pl.bitmap_words;
     a->chunk = pl.chunk; a->n_split = pl.n_split;
+    a->n_items = (int)pl.grid;
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
 }

@@ -1,0 +1,127 @@
+// Shared by all kernels: the argument block, element types, cache addressing, small PTX wrappers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "dsa_mask.cuh"
+
+namespace dsa {
+
+constexpr int NT = 128;          // compute threads per block (4 warps)
+constexpr int MAX_CHUNK = 1024;  // kept rows one work item can hold in its row list
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+struct AttnArgs {
+    const void* q;
+    const void* k;
+    const void* v;
+    int64_t stride_b, stride_tok, stride_head;
+    const int* seq_len;
+    int* seq_len_rw;             // same array, for the append call that advances it
+    const int* prompt_len;
+    const int* block_table;
+    int max_blocks, block_size, num_blocks;
+    int max_seq_len;
+    int ring_size, ring_sinks;   // bounded cache: decode tokens beyond the first ring_sinks live in a ring
+    int B, H_q, H_kv;
+    float scale_log2;            // sm_scale * log2(e)
+    MaskArgs mask;
+    int chunk;                   // kept rows per split (multiple of the tile, <= MAX_CHUNK)
+    int n_split;
+    int n_items;                 // B * H_kv * n_split work items
+    int ring_slots;              // persistent kernel: tiles in its shared-memory ring
+    void* out;                   // n_split == 1: [B, H_q, D] in T
+    float* lse;                  //               [B, H_q]
+    float* out_part;             // n_split > 1:  [B, H_q, n_split, D]
+    float* lse_part;             //               [B, H_q, n_split]
+    // phase-2 selection with n_split > 1: per-split candidates, reduced by the combine kernel
+    float* sel_val_part;         // [B, H_q, n_split] lowest logit (base 2) among this split's candidates
+    int* sel_off_part;           // [B, H_q, n_split] its distance behind the query, -1 if none
+    int* sel_k;                  // [B, H_q] trace entry to write, -1 if this request selects nothing
+    int* error_flag;             // persistent kernel: set if a bounded wait ran out
+};
+
+// Where token `pos` (logical cache position) of request b lives, as an element offset of its kv
+// head 0.  With a bounded cache (ring_size > 0) the prompt and the first ring_sinks decode tokens
+// are stored in order and every later decode token j sits in ring slot (j - ring_sinks) mod
+// ring_size behind them: the slot of the token it evicted ring_size steps earlier.
+__device__ __forceinline__ int64_t token_offset(const AttnArgs& a, int b, int L_p, int pos) {
+    if (a.ring_size > 0) {
+        const int first = L_p + a.ring_sinks;
+        if (pos >= first) pos = first + (pos - first) % a.ring_size;
+    }
+    if (a.block_table) {
+        const int bi = pos / a.block_size;
+        int blk = a.block_table[(int64_t)b * a.max_blocks + min(bi, a.max_blocks - 1)];
+        blk = max(0, min(blk, a.num_blocks - 1));
+        return (int64_t)blk * a.stride_b + (int64_t)(pos - bi * a.block_size) * a.stride_tok;
+    }
+    return (int64_t)b * a.stride_b + (int64_t)pos * a.stride_tok;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int VEC = 8;
+    __device__ static __forceinline__ void unpack(const uint4& r, float (&f)[8]) {
+        const unsigned w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    __device__ static __forceinline__ void store(void* base, int64_t i, float x) {
+        reinterpret_cast<__nv_bfloat16*>(base)[i] = __float2bfloat16_rn(x);
+    }
+};
+template <> struct Elem<float> {
+    static constexpr int VEC = 4;
+    __device__ static __forceinline__ void unpack(const uint4& r, float (&f)[4]) {
+        f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+    __device__ static __forceinline__ void store(void* base, int64_t i, float x) {
+        reinterpret_cast<float*>(base)[i] = x;
+    }
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Sum V values per lane across the LPR lanes of a group; on return every lane holds all V sums.
+// Halving exchange: at each step a lane hands half of its values to its partner and keeps the
+// other half, so V values cost V - 1 + log2(LPR / V) shuffles instead of V * log2(LPR); a final
+// V shuffles hand every sum to every lane.
+template <int V, int LPR>
+__device__ __forceinline__ void group_sum_all(float (&x)[V], int lr) {
+    static_assert(V <= LPR && (V & (V - 1)) == 0, "V must be a power of two <= LPR");
+    constexpr unsigned FULL = 0xffffffffu;
+    int k = 0;
+#pragma unroll
+    for (int off = LPR / 2; off >= 1; off >>= 1, ++k) {
+        const int cnt = (V >> k) > 1 ? (V >> k) : 1;
+        if (cnt > 1) {
+            const int half = cnt / 2;
+            const bool up = (lr & off) != 0;
+#pragma unroll
+            for (int j = 0; j < half; ++j) {
+                const float send = up ? x[j] : x[j + half];
+                const float keep = up ? x[j + half] : x[j];
+                x[j] = keep + __shfl_xor_sync(FULL, send, off);
+            }
+        } else {
+            x[0] += __shfl_xor_sync(FULL, x[0], off);
+        }
+    }
+    // lane lr now holds the sum of value lr / (LPR / V) in x[0]
+    const float mine = x[0];
+#pragma unroll
+    for (int v = 0; v < V; ++v) x[v] = __shfl_sync(FULL, mine, v * (LPR / V), LPR);
+}
+
+}  // namespace dsa

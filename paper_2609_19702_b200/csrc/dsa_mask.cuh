@@ -132,8 +132,18 @@ __device__ __forceinline__ unsigned keep_bits(const MaskArgs& a, const ReqMask& 
     return bits;
 }
 
-// Exclusive scan of one int per thread over a block of NT threads (NT a multiple of 32).
-template <int NT>
+// How the NT threads that build a list wait for each other: the whole block, or (in the persistent
+// kernel, where a loader warp runs beside them) a named barrier over the compute warps only.
+struct BlockSync {
+    __device__ static __forceinline__ void sync() { __syncthreads(); }
+};
+template <int NTHREADS>
+struct NamedSync {
+    __device__ static __forceinline__ void sync() { asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory"); }
+};
+
+// Exclusive scan of one int per thread over NT threads (threadIdx.x < NT, NT a multiple of 32).
+template <int NT, class Sync>
 __device__ __forceinline__ int block_excl_scan(int v, int& total, int* s_warp /* [NT/32] */) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int incl = v;
@@ -142,9 +152,9 @@ __device__ __forceinline__ int block_excl_scan(int v, int& total, int* s_warp /*
         const int n = __shfl_up_sync(0xffffffffu, incl, off);
         if (lane >= off) incl += n;
     }
-    __syncthreads();                      // s_warp may still be read from a previous use
+    Sync::sync();                         // s_warp may still be read from a previous use
     if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
+    Sync::sync();
     int base = 0, tot = 0;
 #pragma unroll
     for (int w = 0; w < NT / 32; ++w) {
@@ -159,8 +169,8 @@ __device__ __forceinline__ int block_excl_scan(int v, int& total, int* s_warp /*
 // Enumerate the kept positions with union rank in [r0, r1), calling
 //   sink(rank - r0, cache position, head bits)
 // for each, and return the total number of kept positions (union over the SLOTS masks).
-// All NT threads of the block must call it (it synchronises).
-template <int NT, int SLOTS, class Sink>
+// All NT threads must call it (it synchronises through Sync).
+template <int NT, int SLOTS, class Sync, class Sink>
 __device__ __forceinline__ int enumerate_kept(const MaskArgs& a, const ReqMask& m,
                                               const unsigned* bitmaps, int r0, int r1,
                                               int* s_warp, Sink sink) {
@@ -184,7 +194,7 @@ __device__ __forceinline__ int enumerate_kept(const MaskArgs& a, const ReqMask& 
     int cnt = 0;
     for (int c = c0; c < c1; ++c) cnt += bits_at(c) != 0u;
     int total;
-    int rank = m.prefix + block_excl_scan<NT>(cnt, total, s_warp);
+    int rank = m.prefix + block_excl_scan<NT, Sync>(cnt, total, s_warp);
     if (rank < r1 && rank + cnt > r0) {
         for (int c = c0; c < c1; ++c) {
             const unsigned bits = bits_at(c);
