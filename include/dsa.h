@@ -111,9 +111,6 @@ typedef struct dsa_problem {
      * tokens per request instead of max_seq_len. */
     int32_t ring_size;
     int32_t ring_sinks;
-    int32_t kernel;            /* 0 = library chooses; 1 = one thread block per work item (cp.async   */
-                               /* ring); 2 = persistent blocks with a loader warp (bulk-copy ring).  */
-                               /* Same results either way; for tests and tuning                       */
 } dsa_problem;
 
 /*
@@ -176,24 +173,13 @@ typedef struct dsa_plan_info {
     int32_t grid_blocks;    /* thread blocks of the attention kernel                               */
     int32_t smem_bytes;     /* dynamic shared memory per block                                     */
     int32_t tile_tokens;    /* tokens per staged K/V tile                                          */
-    int32_t stages;         /* tiles in flight per block (ring slots)                              */
-    int32_t kernel;         /* 1 or 2, see dsa_problem.kernel                                      */
-    int32_t work_items;     /* (request, kv head, split) items; = grid_blocks for kernel 1         */
+    int32_t stages;         /* tiles in flight per block                                           */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);
 DSA_API const char *dsa_status_string(int32_t status);
 /* CUDA error code recorded by the last failing call of this thread (0 if none). */
 DSA_API int32_t dsa_last_cuda_error(void);
-
-/*
- * Kernel 2 bounds every wait inside the kernel; a wait that runs out (which would mean a bug or a
- * broken device, not bad arguments) records a non-zero code in a device-side flag instead of
- * hanging, and the results of that launch are garbage.  This reads the flag of the current
- * device (0 = never happened).  It synchronises with the device: a debugging aid, not part of
- * the hot path.
- */
-DSA_API int32_t dsa_read_device_error(int32_t *code);
 
 /* Bytes of workspace the attention calls need for `problem` (diag == NULL: dense call). */
 DSA_API int32_t dsa_workspace_size(const dsa_problem *problem, const dsa_diag_params *diag, size_t *bytes);

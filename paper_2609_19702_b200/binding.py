@@ -23,7 +23,7 @@ DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
 EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_workspace_size",
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
            "dsa_combine_splits", "dsa_debug_kept_indices",
-           "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_read_device_error"]
+           "dsa_decode_attention_static_scratch", "dsa_append_kv"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -38,8 +38,7 @@ class dsa_problem(ctypes.Structure):
                 ("max_blocks", ctypes.c_int32), ("block_size", ctypes.c_int32),
                 ("num_blocks", ctypes.c_int32), ("max_seq_len", ctypes.c_int32),
                 ("max_prompt_len", ctypes.c_int32), ("split_tokens", ctypes.c_int32),
-                ("ring_size", ctypes.c_int32), ("ring_sinks", ctypes.c_int32),
-                ("kernel", ctypes.c_int32)]
+                ("ring_size", ctypes.c_int32), ("ring_sinks", ctypes.c_int32)]
 
 
 class dsa_diag_params(ctypes.Structure):
@@ -54,7 +53,7 @@ class dsa_plan_info(ctypes.Structure):
     _fields_ = [("split_tokens", ctypes.c_int32), ("n_split", ctypes.c_int32),
                 ("launches", ctypes.c_int32), ("grid_blocks", ctypes.c_int32),
                 ("smem_bytes", ctypes.c_int32), ("tile_tokens", ctypes.c_int32),
-                ("stages", ctypes.c_int32), ("kernel", ctypes.c_int32), ("work_items", ctypes.c_int32)]
+                ("stages", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -79,8 +78,6 @@ def _load() -> ctypes.CDLL:
     lib.dsa_combine_splits.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp]
     lib.dsa_decode_attention_static_scratch.restype = i32
     lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
-    lib.dsa_read_device_error.restype = i32
-    lib.dsa_read_device_error.argtypes = [ctypes.POINTER(ctypes.c_int32)]
     lib.dsa_append_kv.restype = i32
     lib.dsa_append_kv.argtypes = [vp, vp, vp, i32, vp]
     lib.dsa_debug_kept_indices.restype = i32
@@ -142,7 +139,6 @@ class Problem:
     split_tokens: int = 0
     ring_size: int = 0                    # > 0: bounded cache, decode tokens live in a ring
     ring_sinks: int = 0
-    kernel: int = 0                       # 0 auto, 1 block per item, 2 persistent
 
     def c_struct(self) -> dsa_problem:
         b, hq, d = self.q.shape
@@ -165,7 +161,6 @@ class Problem:
         p.max_prompt_len = int(self.max_prompt_len)
         p.split_tokens = int(self.split_tokens)
         p.ring_size, p.ring_sinks = int(self.ring_size), int(self.ring_sinks)
-        p.kernel = int(self.kernel)
         return p
 
 
@@ -201,13 +196,6 @@ def _ref(s):
 
 def dsa_version() -> int:
     return int(_lib.dsa_version())
-
-
-def dsa_read_device_error() -> int:
-    """Code left by a persistent kernel whose bounded wait ran out (0 = none).  Synchronises."""
-    code = ctypes.c_int32(0)
-    _check("dsa_read_device_error", _lib.dsa_read_device_error(ctypes.byref(code)))
-    return int(code.value)
 
 
 def dsa_workspace_size(problem: Problem, diag: Optional[Diag] = None) -> int:
@@ -312,7 +300,7 @@ def dsa_debug_kept_indices(problem: Problem, diag: Optional[Diag], max_kept: int
 
 
 def problem_from_host(inp: dict, device: str = "cuda", dtype: torch.dtype = torch.bfloat16,
-                      split_tokens: int = 0, kernel: int = 0) -> Problem:
+                      split_tokens: int = 0) -> Problem:
     """Copy one host batch (as made by ``synth.make_inputs``: bf16 bit patterns) to the device."""
     w = inp["workload"]
 
@@ -329,4 +317,4 @@ def problem_from_host(inp: dict, device: str = "cuda", dtype: torch.dtype = torc
         num_kv_heads=w.num_kv_heads, max_seq_len=inp["max_seq_len"], max_prompt_len=w.prompt_len,
         block_table=None if bt is None else torch.from_numpy(bt).to(device),
         block_size=inp["block_size"], num_blocks=0 if bt is None else int(bt.size),
-        split_tokens=split_tokens, kernel=kernel)
+        split_tokens=split_tokens)

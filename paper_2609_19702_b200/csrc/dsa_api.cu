@@ -5,10 +5,7 @@
 #include <cmath>
 #include <cstdio>
 
-#include <cstdlib>
-
 #include "dsa_attn.cuh"
-#include "dsa_attn_persistent.cuh"
 
 namespace {
 
@@ -23,29 +20,6 @@ int32_t cuda_fail(cudaError_t e) {
 
 constexpr int kNumSMs = 148;
 constexpr int kMaxDevices = 64;
-constexpr int kSmemPerSM = 227 * 1024;
-
-// Set by a persistent kernel whose bounded wait ran out (0 = never happened).
-__device__ int g_device_error = 0;
-
-int* device_error_ptr(cudaError_t* err) {
-    static int* ptr[kMaxDevices] = {};
-    int dev = 0;
-    *err = cudaGetDevice(&dev);
-    if (*err != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    if (!ptr[dev]) {
-        void* p = nullptr;
-        *err = cudaGetSymbolAddress(&p, g_device_error);
-        if (*err != cudaSuccess) return nullptr;
-        ptr[dev] = static_cast<int*>(p);
-    }
-    return ptr[dev];
-}
-
-int env_int(const char* name, int fallback) {
-    const char* v = std::getenv(name);
-    return (v && *v) ? std::atoi(v) : fallback;
-}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -58,9 +32,6 @@ struct Plan {
     int tile, stages;
     int chunk, n_split;
     int bitmap_words;
-    int kernel;          // 1: one block per work item; 2: persistent blocks with a loader warp
-    int ring_slots;      // kernel 2: tiles in the shared-memory ring
-    int persist_grid;    // kernel 2: blocks launched
     int64_t grid;
     size_t smem;
     size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
@@ -86,25 +57,7 @@ struct KernelPick {
     static constexpr int STAGES = kStagesDefault;
 #endif
     using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM, SEL>;
-    using PCfg = PersistCfg<T, D, G, TILE, HM, SEL>;
     static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
-    static size_t persist_fixed(int chunk, int bw) { return PCfg::fixed_bytes(chunk, bw); }
-    static size_t persist_smem(int slots, int chunk, int bw) { return PCfg::smem_bytes(slots, chunk, bw); }
-    static constexpr int kSlotBytes = PCfg::SLOT_BYTES + 16;
-    static cudaError_t launch_persistent(const AttnArgs& a, int grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_persistent_kernel<T, D, G, TILE, HM, SEL>;
-        static bool configured[kMaxDevices] = {};
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
-        }
-        kern<<<(unsigned)grid, NT_PERSIST, smem_bytes, st>>>(a);
-        return cudaGetLastError();
-    }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
         auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
         static bool configured[kMaxDevices] = {};
@@ -172,7 +125,6 @@ int32_t check_problem(const dsa_problem* p) {
     if (p->stride_batch < 0 || p->stride_token < p->head_dim || p->stride_head < 0) return DSA_ERR_INVALID_ARG;
     if (p->stride_batch % vec || p->stride_token % vec || p->stride_head % vec) return DSA_ERR_INVALID_ARG;
     if (p->ring_size < 0 || p->ring_sinks < 0) return DSA_ERR_INVALID_ARG;
-    if (p->kernel < 0 || p->kernel > 2) return DSA_ERR_INVALID_ARG;
     if (p->ring_size > 0 && p->max_prompt_len < 1) return DSA_ERR_INVALID_ARG;   // capacity needs the bound
     if (p->block_table) {
         if (p->block_size < 1 || p->max_blocks < 1 || p->num_blocks < 1) return DSA_ERR_INVALID_ARG;
@@ -268,36 +220,6 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->smem = smem_probe;
     if (pl->smem > 200 * 1024) return DSA_ERR_UNSUPPORTED;     // window too large for LIST bitmaps
 
-    // Which kernel.  The persistent one keeps `ctas` blocks per SM, each with as many ring slots as
-    // its share of the shared memory holds.  (DSA_PERSIST_CTAS / DSA_PERSIST_SLOTS / DSA_KERNEL are
-    // tuning overrides read from the environment.)
-    pl->kernel = p->kernel ? p->kernel : env_int("DSA_KERNEL", 1);
-    pl->ring_slots = 0;
-    pl->persist_grid = 0;
-    if (pl->kernel == 2) {
-        const int ctas = std::max(1, std::min(8, env_int("DSA_PERSIST_CTAS", 3)));
-        size_t fixed = 0;
-        int slot_bytes = 1;
-        dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
-            using P = decltype(pick);
-            fixed = P::persist_fixed(pl->chunk, pl->bitmap_words);
-            slot_bytes = P::kSlotBytes;
-            return DSA_OK;
-        });
-        const long long budget = (long long)kSmemPerSM / ctas - 1024 - 64 - (long long)fixed;
-        int slots = (int)std::min<long long>(64, budget / slot_bytes);
-        slots = env_int("DSA_PERSIST_SLOTS", slots);
-        if (slots < 2) return DSA_ERR_UNSUPPORTED;
-        pl->ring_slots = slots;
-        dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
-            using P = decltype(pick);
-            pl->smem = P::persist_smem(slots, pl->chunk, pl->bitmap_words);
-            return DSA_OK;
-        });
-        if (pl->smem > 200 * 1024) return DSA_ERR_UNSUPPORTED;
-        pl->persist_grid = (int)std::min<int64_t>(pl->grid, (int64_t)ctas * kNumSMs);
-    }
-
     if (pl->n_split > 1) {
         const size_t rows = (size_t)p->batch * p->num_q_heads * pl->n_split;
         pl->ws_out_bytes = (rows * p->head_dim * sizeof(float) + 255) / 256 * 256;
@@ -338,7 +260,6 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.bitmap_words = pl.bitmap_words;
     a->chunk = pl.chunk; a->n_split = pl.n_split;
     a->n_items = (int)pl.grid;
-    a->ring_slots = pl.ring_slots;
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
 }
@@ -385,14 +306,9 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    if (pl.kernel == 2) {
-        a.error_flag = device_error_ptr(&err);
-        if (err != cudaSuccess) return cuda_fail(err);
-    }
     rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, pl.select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
-        err = pl.kernel == 2 ? P::launch_persistent(a, pl.persist_grid, pl.smem, st)
-                             : P::launch(a, pl.grid, pl.smem, st);
+        err = P::launch(a, pl.grid, pl.smem, st);
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;
@@ -423,15 +339,6 @@ const char* dsa_status_string(int32_t status) {
 
 int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
 
-int32_t dsa_read_device_error(int32_t* code) {
-    if (!code) return DSA_ERR_INVALID_ARG;
-    int v = 0;
-    const cudaError_t e = cudaMemcpyFromSymbol(&v, g_device_error, sizeof(int));
-    if (e != cudaSuccess) return cuda_fail(e);
-    *code = v;
-    return DSA_OK;
-}
-
 int32_t dsa_workspace_size(const dsa_problem* problem, const dsa_diag_params* diag, size_t* bytes) {
     if (!bytes) return DSA_ERR_INVALID_ARG;
     Plan pl;
@@ -449,12 +356,10 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->split_tokens = pl.chunk;
     info->n_split = pl.n_split;
     info->launches = problem->batch == 0 ? 0 : (pl.n_split > 1 ? 2 : 1);
-    info->grid_blocks = pl.kernel == 2 ? pl.persist_grid : (int32_t)pl.grid;
-    info->kernel = pl.kernel;
-    info->work_items = (int32_t)pl.grid;
+    info->grid_blocks = (int32_t)pl.grid;
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;
-    info->stages = pl.kernel == 2 ? pl.ring_slots : pl.stages;
+    info->stages = pl.stages;
     return DSA_OK;
 }
 

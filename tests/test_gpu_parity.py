@@ -33,12 +33,11 @@ def _run_gpu(dsa, prob, diag):
 
 
 def _check_all_modes(dsa, inp, *, f32=False, split_tokens=0, list_heads=(1,), seed=0, what="",
-                     max_prompt_len=None, kernel=0):
+                     max_prompt_len=None):
     """Dense, window-only, grid and list masks of one host batch against the oracle."""
     w = inp["workload"]
     dtype = torch.float32 if f32 else torch.bfloat16
-    prob = dsa.problem_from_host(inp, dtype=dtype, split_tokens=split_tokens, kernel=kernel)
-    what = what + " kernel %d" % kernel
+    prob = dsa.problem_from_host(inp, dtype=dtype, split_tokens=split_tokens)
     if max_prompt_len is not None:
         prob.max_prompt_len = max_prompt_len
     s_max = inp["max_seq_len"]
@@ -90,18 +89,13 @@ def _check_all_modes(dsa, inp, *, f32=False, split_tokens=0, list_heads=(1,), se
 
 # ---------------------------------------------------------------- the five configurations
 
-KERNELS = [1, 2]       # one block per work item / persistent blocks with a loader warp
-
-
-@pytest.mark.parametrize("kernel", KERNELS)
-def test_config1_every_position(dsa, kernel):
+def test_config1_every_position(dsa):
     # 16x16 grid, one query at every image position 1..256, all sharing one cache
     w = synth.workload(1)
     inp = synth.make_inputs(w)
     assert inp["position"].tolist() == list(range(1, 257))
-    _check_all_modes(dsa, inp, list_heads=(1, 8), what="config1", kernel=kernel)
-    _check_all_modes(dsa, inp, f32=True, list_heads=(8,), what="config1 f32", kernel=kernel)
-    assert dsa.dsa_read_device_error() == 0
+    _check_all_modes(dsa, inp, list_heads=(1, 8), what="config1")
+    _check_all_modes(dsa, inp, f32=True, list_heads=(8,), what="config1 f32")
 
 
 def test_config1_paper_trace_from_oracle_argmin(dsa):
@@ -120,13 +114,12 @@ def test_config1_paper_trace_from_oracle_argmin(dsa):
     assert torch.equal(c1, c2) and torch.equal(i1, i2)
 
 
-@pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("index", [2, 3, 4])
-def test_configs_2_3_4(dsa, index, kernel):
+def test_configs_2_3_4(dsa, index):
     w = synth.workload(index)
     inp = synth.make_inputs(w)
     heads = (w.num_q_heads,) if index == 4 else (1,)
-    _check_all_modes(dsa, inp, list_heads=heads, seed=index, what="config%d" % index, kernel=kernel)
+    _check_all_modes(dsa, inp, list_heads=heads, seed=index, what="config%d" % index)
 
 
 @pytest.mark.parametrize("batch", [1, 8])
@@ -134,9 +127,7 @@ def test_config5_paged_small_batches(dsa, batch):
     for window, n_att in ((512, 208), (1024, 416)):
         w = synth.workload(5, batch=batch, window=window, n_att=n_att)
         inp = synth.make_inputs(w)
-        for kernel in KERNELS:
-            _check_all_modes(dsa, inp, list_heads=(w.num_q_heads,), seed=batch, what="config5 B=%d" % batch,
-                             kernel=kernel)
+        _check_all_modes(dsa, inp, list_heads=(w.num_q_heads,), seed=batch, what="config5 B=%d" % batch)
 
 
 # ---------------------------------------------------------------- properties on small shapes
@@ -152,10 +143,9 @@ SMALL = [
 ]
 
 
-@pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("case", range(len(SMALL)))
 @pytest.mark.parametrize("f32", [False, True])
-def test_small_shapes_all_masks_and_splits(dsa, case, f32, kernel):
+def test_small_shapes_all_masks_and_splits(dsa, case, f32):
     hq, hkv, d, l_p, gh, gw, extra, n_r, n_att, paged, bs = SMALL[case]
     w = synth.Workload("small%d" % case, 10 + case, 7, hq, hkv, d, l_p, gh, gw, extra, n_r, n_att,
                        1, gh * (gw + extra), positional=bool(case % 2), paged=paged, block_size=bs)
@@ -163,8 +153,7 @@ def test_small_shapes_all_masks_and_splits(dsa, case, f32, kernel):
     heads = sorted({1, hkv, hq})
     for split in (0, 32, 96, 1024):
         _check_all_modes(dsa, inp, f32=f32, split_tokens=split, list_heads=heads, seed=case,
-                         what="small%d split=%d" % (case, split), kernel=kernel)
-    assert dsa.dsa_read_device_error() == 0
+                         what="small%d split=%d" % (case, split))
 
 
 def test_split_counts_agree(dsa):
@@ -195,10 +184,8 @@ def test_degenerate_requests(dsa):
     inp["prompt_len"][2] = 0                    # no prompt
     inp["seq_len"][2] = 3
     inp["prompt_len"][3] = inp["seq_len"][3] + 5  # prompt_len above seq_len reads as seq_len
-    for kernel in KERNELS:
-        _check_all_modes(dsa, inp, list_heads=(1, 4), what="degenerate", max_prompt_len=0, kernel=kernel)
-        _check_all_modes(dsa, inp, split_tokens=32, list_heads=(2,), what="degenerate split", max_prompt_len=0,
-                         kernel=kernel)
+    _check_all_modes(dsa, inp, list_heads=(1, 4), what="degenerate", max_prompt_len=0)
+    _check_all_modes(dsa, inp, split_tokens=32, list_heads=(2,), what="degenerate split", max_prompt_len=0)
 
 
 def test_empty_batch_and_bad_arguments(dsa):
