@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdsa.so")
 SOURCES = ["dsa_api.cu"]
-HEADERS = ["dsa_attn.cuh", "dsa_tile.cuh", "dsa_common.cuh", "dsa_mask.cuh",
+HEADERS = ["dsa_attn.cuh", "dsa_attn_mma.cuh", "dsa_tile.cuh", "dsa_common.cuh", "dsa_mask.cuh",
            os.path.join("..", "..", "include", "dsa.h")]
 
 

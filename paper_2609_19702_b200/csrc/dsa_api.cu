@@ -5,7 +5,10 @@
 #include <cmath>
 #include <cstdio>
 
+#include <cstdlib>
+
 #include "dsa_attn.cuh"
+#include "dsa_attn_mma.cuh"
 
 namespace {
 
@@ -20,6 +23,15 @@ int32_t cuda_fail(cudaError_t e) {
 
 constexpr int kNumSMs = 148;
 constexpr int kMaxDevices = 64;
+#ifndef DSA_TUNE_MMA_STAGES
+#define DSA_TUNE_MMA_STAGES 3
+#endif
+constexpr int kMmaStages = DSA_TUNE_MMA_STAGES;    // 16-key tiles in flight per warp (+1 being consumed)
+
+int env_int(const char* name, int fallback) {
+    const char* v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : fallback;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -32,6 +44,8 @@ struct Plan {
     int tile, stages;
     int chunk, n_split;
     int bitmap_words;
+    bool mma;            // bf16: one warp per work item, tensor-core tiles
+    int mma_warps;       // warps (= kv heads) per block that share one row list
     int64_t grid;
     size_t smem;
     size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
@@ -58,6 +72,43 @@ struct KernelPick {
 #endif
     using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM, SEL>;
     static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
+    // Tensor-core kernel (bf16 only).  W warps per block share one row list when the mask does not
+    // depend on the head (never with per-head masks or selection).
+    template <int W>
+    static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, kMmaStages, HM, SEL, W>::smem_bytes(chunk, bw); }
+    static size_t smem_mma(int w, int chunk, int bw) {
+        if constexpr (!HM && !SEL) {
+            if (w == 4) return smem_mma_w<4>(chunk, bw);
+            if (w == 2) return smem_mma_w<2>(chunk, bw);
+        }
+        return smem_mma_w<1>(chunk, bw);
+    }
+    template <int W>
+    static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
+        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W>;
+        static bool configured[kMaxDevices] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        }
+        kern<<<(unsigned)grid, 32 * W, smem_bytes, st>>>(a);
+        return cudaGetLastError();
+    }
+    static cudaError_t launch_mma(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
+        if constexpr (sizeof(T) == 2) {
+            if constexpr (!HM && !SEL) {
+                if (w == 4) return launch_mma_w<4>(a, items / 4, smem_bytes, st);
+                if (w == 2) return launch_mma_w<2>(a, items / 2, smem_bytes, st);
+            }
+            return launch_mma_w<1>(a, items, smem_bytes, st);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
         auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
         static bool configured[kMaxDevices] = {};
@@ -191,6 +242,17 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;
+    // bf16 runs on the tensor-core kernel (one warp per work item); fp32 on the CUDA-core kernel.
+    // DSA_CUDA_CORES=1 forces the latter for bf16 too (comparison runs).
+    pl->mma = p->dtype == DSA_BF16 && env_int("DSA_CUDA_CORES", 0) == 0;
+    pl->mma_warps = 1;
+    if (pl->mma) {
+        pl->tile = MMA_KEYS;
+        pl->stages = kMmaStages;
+        const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
+        if (shared_mask) pl->mma_warps = p->num_kv_heads % 4 == 0 ? 4 : (p->num_kv_heads % 2 == 0 ? 2 : 1);
+        pl->mma_warps = std::min(pl->mma_warps, std::max(1, env_int("DSA_MMA_WARPS", 2)));
+    }
 
     int chunk;
     if (p->split_tokens > 0) {
@@ -200,9 +262,9 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         // split only while fewer than ~4 blocks per SM exist, never below 128 rows per block, and
         // balance the splits (equal chunks rather than full ones plus a short tail).
         const int64_t pairs = (int64_t)std::max(p->batch, 1) * p->num_kv_heads;
-        const int64_t target = 4 * kNumSMs;
+        const int64_t target = (pl->mma ? 6 : 4) * kNumSMs;        // a work item is a warp / a 4-warp block
         int64_t want_split = std::max<int64_t>(1, (target + pairs - 1) / pairs);
-        want_split = std::min<int64_t>(want_split, std::max<int64_t>(1, bound / 128));
+        want_split = std::min<int64_t>(want_split, std::max<int64_t>(1, bound / (pl->mma ? 96 : 128)));
         want_split = std::max<int64_t>(want_split, (bound + MAX_CHUNK - 1) / MAX_CHUNK);
         const int64_t c = (bound + want_split - 1) / want_split;
         chunk = std::min(MAX_CHUNK, round_up((int)c, pl->tile));
@@ -214,7 +276,8 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
 
     dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
-        smem_probe = P::smem(pl->chunk, pl->bitmap_words);
+        smem_probe = pl->mma ? P::smem_mma(pl->mma_warps, pl->chunk, pl->bitmap_words)
+                             : P::smem(pl->chunk, pl->bitmap_words);
         return DSA_OK;
     });
     pl->smem = smem_probe;
@@ -308,7 +371,7 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     cudaError_t err = cudaSuccess;
     rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, pl.select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
-        err = P::launch(a, pl.grid, pl.smem, st);
+        err = pl.mma ? P::launch_mma(pl.mma_warps, a, pl.grid, pl.smem, st) : P::launch(a, pl.grid, pl.smem, st);
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;
@@ -356,7 +419,7 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->split_tokens = pl.chunk;
     info->n_split = pl.n_split;
     info->launches = problem->batch == 0 ? 0 : (pl.n_split > 1 ? 2 : 1);
-    info->grid_blocks = (int32_t)pl.grid;
+    info->grid_blocks = (int32_t)(pl.mma ? pl.grid / pl.mma_warps : pl.grid);
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;
     info->stages = pl.stages;

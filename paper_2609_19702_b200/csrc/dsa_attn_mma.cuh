@@ -1,0 +1,296 @@
+// Split-KV decode attention for bf16 caches: ONE WARP per work item, tensor-core tiles.
+//
+// Why tensor cores in a bandwidth-bound kernel: with fp32 FMAs on the CUDA cores the scan costs
+// about 0.14 warp instructions per byte; at 6.5-7 TB/s that is 80-90 % of the issue slots of the
+// 148 SMs (measured), i.e. the kernel had become issue-bound.  mma.sync m16n8k16 brings it to
+// about 0.02 instructions per byte; that most of each MMA multiplies padding is irrelevant.
+//
+// Formulation (transposed, so that the 16-row MMA dimension is filled with keys, not heads):
+//   S^T[16 keys x 8 heads]  = K_tile[16 keys x D] . Q^T[D x 8 heads]          (D/16 MMAs)
+//   O^T[D x 8 heads]       += V_tile^T[D x 16 keys] . P^T[16 keys x 8 heads]   (D/16 MMAs)
+// The 8 "heads" are the G <= 8 query heads that share this kv head (GQA packing), the rest zero.
+// K is the row-major A operand (ldmatrix), V^T comes from ldmatrix.trans on the same [key][dim]
+// layout, P^T is moved from accumulator layout to B-operand layout with movmatrix.  Online
+// softmax runs on the accumulator fragment: a thread owns two head columns and keys lane/4 and
+// lane/4 + 8; column maxima take three shuffles, sums are kept per thread and reduced once.
+//
+// A work item belongs to a single warp, which streams it through its own 2-3 stage cp.async ring of
+// 16-key tiles: no block barrier in the main loop, the hardware schedules and balances the warps,
+// and ~10 of them per SM keep well over 100 KB in flight.  A block holds W warps that work on W
+// neighbouring kv heads of the same (request, split): whenever the mask does not depend on the
+// head (dense, window, grid, one shared list) the row list is the same for all of them, so the
+// block builds it once with all its threads and every warp only adds its head's offset.  Masks
+// per head run with W = 1.  Shared-memory tiles are XOR-swizzled in 16-byte chunks so that the
+// ldmatrix row reads are conflict-free.
+#pragma once
+#include "dsa_tile.cuh"
+
+namespace dsa {
+
+constexpr int MMA_KEYS = 16;     // keys per tile
+
+__device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], const void* smem_row) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"((unsigned)__cvta_generic_to_shared(smem_row)));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], const void* smem_row) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"((unsigned)__cvta_generic_to_shared(smem_row)));
+}
+__device__ __forceinline__ unsigned movmatrix_trans(unsigned x) {
+    unsigned y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// {lo, hi} -> packed bf16x2 (lo in the low half)
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
+    unsigned d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ void cp_async16_w(void* smem_dst, const void* gmem_src, bool valid) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    const int src_size = valid ? 16 : 0;     // 0: nothing is read, the 16 bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_size));
+}
+
+template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W = 1>
+struct MmaCfg {
+    using T = __nv_bfloat16;
+    static constexpr int ROW_BYTES = D * 2;
+    static constexpr int CPR = ROW_BYTES / 16;              // 16-byte chunks per row (8 or 16)
+    static constexpr int TILE_BYTES = MMA_KEYS * ROW_BYTES; // one K (or V) tile
+    static constexpr int SLOT_BYTES = 2 * TILE_BYTES;
+    static constexpr int KSTEPS = D / 16;                   // MMAs of the score product
+    static constexpr int MTILES = D / 16;                   // MMAs of the output product
+    static constexpr int SLOTS = HEADMASK ? G : 1;
+    __host__ __device__ static constexpr int list_bytes(int chunk) {
+        return chunk * 8 + (SELECT ? chunk * 4 : 0) + (HEADMASK ? ((chunk + 15) / 16) * 16 : 0);
+    }
+    // dynamic shared memory: [W rings: STAGES x (K tile, V tile)][row list][bitmaps]
+    __host__ static size_t smem_bytes(int chunk, int bitmap_words) {
+        return (size_t)W * STAGES * SLOT_BYTES + list_bytes(chunk) + (size_t)SLOTS * bitmap_words * 4;
+    }
+};
+
+// adapter with the member names the shared list-building code uses
+template <int D_, int G_, bool HEADMASK_, bool SELECT_>
+struct MmaItemCfg {
+    using T = __nv_bfloat16;
+    static constexpr int D = D_, G = G_;
+    static constexpr bool HEADMASK = HEADMASK_, SELECT = SELECT_;
+    static constexpr int SLOTS = HEADMASK ? G : 1;
+};
+
+template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W>
+__global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) {
+    using C = MmaCfg<D, G, STAGES, HEADMASK, SELECT, W>;
+    using IC = MmaItemCfg<D, G, HEADMASK, SELECT>;
+    using T = __nv_bfloat16;
+    constexpr unsigned FULL = 0xffffffffu;
+    static_assert(W == 1 || (!HEADMASK && !SELECT), "a shared row list needs a head-independent mask");
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int s_warp[W];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned char* ring = smem + warp * (STAGES * C::SLOT_BYTES);
+    const RowList list = RowList::carve<IC>(smem + W * STAGES * C::SLOT_BYTES, a.chunk);
+    unsigned* bitmaps = reinterpret_cast<unsigned*>(smem + W * STAGES * C::SLOT_BYTES + C::list_bytes(a.chunk));
+
+    // kv heads vary fastest across the grid: the warps that run together read the same tokens
+    // of neighbouring heads, i.e. neighbouring memory.
+    const int hblocks = a.H_kv / W;
+    const int kvh = (blockIdx.x % hblocks) * W + warp;
+    const int split = (blockIdx.x / hblocks) % a.n_split;
+    const int b = blockIdx.x / (hblocks * a.n_split);
+
+    const ReqMask m = req_mask_setup(a.mask, a.seq_len[b], a.prompt_len[b], a.max_seq_len);
+    // W > 1: one list for all the block's heads, built without a head offset (kv head "0")
+    const int n_rows = W == 1 ? build_row_list<IC, WarpSync, 32>(a, m, b, kvh, split, list, bitmaps, s_warp)
+                              : build_row_list<IC, BlockSync, 32 * W>(a, m, b, 0, split, list, bitmaps, s_warp);
+    if (n_rows <= 0) { write_empty_item<IC, 32>(a, m, b, kvh, split, lane); return; }
+    if (W == 1) __syncwarp(); else __syncthreads();     // the last barrier: from here on warps run free
+    const int64_t head_bytes = W == 1 ? 0 : (int64_t)kvh * a.stride_head * 2;
+
+    // ---- staging: this warp's own ring of 16-key tiles ---------------------------------------
+    const int n_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
+    const unsigned char* kbase = reinterpret_cast<const unsigned char*>(a.k);
+    const unsigned char* vbase = reinterpret_cast<const unsigned char*>(a.v);
+    auto issue_tile = [&](int tile) {
+        if (tile < n_tiles) {
+            unsigned char* ks = ring + (tile % STAGES) * C::SLOT_BYTES;
+            unsigned char* vs = ks + C::TILE_BYTES;
+#pragma unroll
+            for (int i = 0; i < MMA_KEYS * C::CPR / 32; ++i) {
+                const int idx = i * 32 + lane;
+                const int row = idx / C::CPR, c = idx % C::CPR;
+                const int r = tile * MMA_KEYS + row;
+                const bool valid = r < n_rows;
+                const int64_t off = valid ? list.rowoff[r] * 2 + head_bytes + c * 16 : 0;
+                const int dst = row * C::ROW_BYTES + ((c ^ (row & 7)) * 16);       // swizzled chunk
+                cp_async16_w(ks + dst, kbase + off, valid);
+                cp_async16_w(vs + dst, vbase + off, valid);
+            }
+        }
+        asm volatile("cp.async.commit_group;\n" ::);
+    };
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) issue_tile(s);
+
+    // ---- Q^T as B operand: head = lane / 4, dims 2*(lane%4)+{0,1} (+8) of every 16-dim step ----
+    const int hq = lane >> 2;                 // head column this thread feeds
+    const int qd = (lane & 3) * 2;
+    unsigned qb[C::KSTEPS][2];
+    {
+        const T* qrow = reinterpret_cast<const T*>(a.q) + ((int64_t)b * a.H_q + kvh * G + (hq < G ? hq : 0)) * D;
+#pragma unroll
+        for (int kk = 0; kk < C::KSTEPS; ++kk) {
+            const unsigned lo = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd);
+            const unsigned hi = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd + 8);
+            qb[kk][0] = hq < G ? lo : 0u;
+            qb[kk][1] = hq < G ? hi : 0u;
+        }
+    }
+    // accumulator-fragment coordinates: keys (or dims) lane/4 and lane/4 + 8, heads hc and hc + 1
+    const int hc = (lane & 3) * 2;
+    const int kr = lane >> 2;
+    float o[C::MTILES][4];
+#pragma unroll
+    for (int mt = 0; mt < C::MTILES; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
+    float mrun[2] = {-INFINITY, -INFINITY}, lpart[2] = {0.f, 0.f};
+    float bestv[2] = {INFINITY, INFINITY};
+    int bestp[2] = {0x7fffffff, 0x7fffffff};
+    const int cand_lo = m.L_p + a.mask.n_sink;
+
+    // per-lane ldmatrix row addresses inside a tile (swizzle applied per k-step / m-tile below)
+    const int lm_row_k = (lane & 7) + ((lane >> 3) & 1) * 8;     // K as A: matrices (r0-7,c0) (r8-15,c0) (r0-7,c1) (r8-15,c1)
+    const int lm_chk_k = lane >> 4;
+    const int lm_row_v = (lane & 7) + (lane >> 4) * 8;           // V^T as A: (k0-7,d0) (k0-7,d1) (k8-15,d0) (k8-15,d1)
+    const int lm_chk_v = (lane >> 3) & 1;
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        asm volatile("cp.async.wait_group %0;\n" ::"n"(STAGES - 2));
+        __syncwarp();                                   // tile landed for every lane; tile-1 fully consumed
+        issue_tile(tile + STAGES - 1);
+        const unsigned char* ks = ring + (tile % STAGES) * C::SLOT_BYTES;
+        const unsigned char* vs = ks + C::TILE_BYTES;
+
+        // S^T = K . Q^T
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int kk = 0; kk < C::KSTEPS; ++kk) {
+            unsigned af[4];
+            const int chunk = kk * 2 + lm_chk_k;
+            ldmatrix_x4(af, ks + lm_row_k * C::ROW_BYTES + ((chunk ^ (lm_row_k & 7)) * 16));
+            mma_bf16_16816(s, af, qb[kk][0], qb[kk][1]);
+        }
+        // s[0]: (key kr, head hc)  s[1]: (kr, hc+1)  s[2]: (kr+8, hc)  s[3]: (kr+8, hc+1)
+        const int r0 = tile * MMA_KEYS + kr, r1 = r0 + 8;
+        const bool v0 = r0 < n_rows, v1 = r1 < n_rows;
+        unsigned bits0 = 0xffu, bits1 = 0xffu;
+        if (HEADMASK) { bits0 = v0 ? list.hbits[r0] : 0u; bits1 = v1 ? list.hbits[r1] : 0u; }
+        int pos0 = 0, pos1 = 0;
+        if (SELECT) { pos0 = v0 ? list.rowpos[r0] : 0; pos1 = v1 ? list.rowpos[r1] : 0; }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {                   // the thread's two head columns
+            const bool on0 = v0 && (!HEADMASK || ((bits0 >> (hc + j)) & 1u));
+            const bool on1 = v1 && (!HEADMASK || ((bits1 >> (hc + j)) & 1u));
+            float x0 = on0 ? s[j] * a.scale_log2 : -INFINITY;
+            float x1 = on1 ? s[2 + j] * a.scale_log2 : -INFINITY;
+            if (SELECT) {
+                // keys arrive in ascending position: a strict "<" keeps the oldest of equal logits
+                if (on0 && pos0 >= cand_lo && x0 < bestv[j]) { bestv[j] = x0; bestp[j] = pos0; }
+                if (on1 && pos1 >= cand_lo && x1 < bestv[j]) { bestv[j] = x1; bestp[j] = pos1; }
+            }
+            float mx = fmaxf(x0, x1);
+            mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 16));
+            const float mnew = fmaxf(mrun[j], mx);
+            const float msafe = mnew == -INFINITY ? 0.f : mnew;
+            const float corr = fast_exp2(mrun[j] - msafe);
+            x0 = fast_exp2(x0 - msafe);
+            x1 = fast_exp2(x1 - msafe);
+            lpart[j] = lpart[j] * corr + x0 + x1;
+            mrun[j] = mnew;
+            s[j] = x0; s[2 + j] = x1;
+            if (corr != 1.f) {
+#pragma unroll
+                for (int mt = 0; mt < C::MTILES; ++mt) { o[mt][j] *= corr; o[mt][2 + j] *= corr; }
+            }
+        }
+        // P^T as B operand: accumulator layout [key][head] -> operand layout [head][key]
+        const unsigned pb0 = movmatrix_trans(pack_bf16x2(s[0], s[1]));     // keys 0-7
+        const unsigned pb1 = movmatrix_trans(pack_bf16x2(s[2], s[3]));     // keys 8-15
+        // O^T += V^T . P^T
+#pragma unroll
+        for (int mt = 0; mt < C::MTILES; ++mt) {
+            unsigned af[4];
+            const int chunk = mt * 2 + lm_chk_v;
+            ldmatrix_x4_trans(af, vs + lm_row_v * C::ROW_BYTES + ((chunk ^ (lm_row_v & 7)) * 16));
+            mma_bf16_16816(o[mt], af, pb0, pb1);
+        }
+    }
+    asm volatile("cp.async.wait_group 0;\n" ::);
+
+    // ---- finish: sums over the key lanes, normalise, write ------------------------------------
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        float l = lpart[j];
+        l += __shfl_xor_sync(FULL, l, 4);
+        l += __shfl_xor_sync(FULL, l, 8);
+        l += __shfl_xor_sync(FULL, l, 16);
+        float bv = bestv[j];
+        int bp = bestp[j];
+        if (SELECT) {
+#pragma unroll
+            for (int off = 4; off <= 16; off <<= 1) {
+                const float ov = __shfl_xor_sync(FULL, bv, off);
+                const int op = __shfl_xor_sync(FULL, bp, off);
+                if (ov < bv || (ov == bv && op < bp)) { bv = ov; bp = op; }
+            }
+        }
+        const int h = hc + j;
+        if (h < G) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            const float lse = l > 0.f ? (mrun[j] + log2f(l)) * LN2 : -INFINITY;
+            const int64_t row = (int64_t)b * a.H_q + kvh * G + h;
+#pragma unroll
+            for (int mt = 0; mt < C::MTILES; ++mt) {
+                const int d0 = mt * 16 + kr;
+                if (a.n_split > 1) {
+                    float* dst = a.out_part + (row * a.n_split + split) * D;
+                    dst[d0] = o[mt][j] * inv;
+                    dst[d0 + 8] = o[mt][2 + j] * inv;
+                } else {
+                    T* dst = reinterpret_cast<T*>(a.out) + row * D;
+                    dst[d0] = __float2bfloat16_rn(o[mt][j] * inv);
+                    dst[d0 + 8] = __float2bfloat16_rn(o[mt][2 + j] * inv);
+                }
+            }
+            if (kr == 0) {
+                if (a.n_split > 1) a.lse_part[row * a.n_split + split] = lse;
+                else a.lse[row] = lse;
+                if (SELECT) {
+                    const int off = bp == 0x7fffffff ? -1 : (m.S - 1) - bp;
+                    if (a.n_split > 1) {
+                        a.sel_val_part[row * a.n_split + split] = bv;
+                        a.sel_off_part[row * a.n_split + split] = off;
+                        a.sel_k[row] = m.sel_k;
+                    } else if (m.sel_k >= 0) {
+                        a.mask.skip_offsets[row * a.mask.trace_len + m.sel_k] = off;
+                    }
+                }
+            }
+        }
+    }
+}
+
+}  // namespace dsa

@@ -96,15 +96,6 @@ __device__ __forceinline__ ReqMask req_mask_setup(const MaskArgs& a, int seq_len
     return m;
 }
 
-__device__ __forceinline__ bool grid_keep(const ReqMask& m, int stride, int o) {
-    if (o == m.T) return true;
-    const int k = o / stride, r = o - k * stride;
-    const int d = min(r, stride - r);
-    if (d != m.dstar) return d < m.dstar;
-    const int rank = (m.dstar == 0 || 2 * m.dstar == stride) ? k : 2 * k + (r == m.dstar ? 0 : 1);
-    return rank < m.need;
-}
-
 // LIST: set the bits of the active skip distances of one trace in a shared-memory bitmap
 // (cleared by the caller).  Distances outside [0, window) are ignored.
 template <int NT>
@@ -116,13 +107,12 @@ __device__ __forceinline__ void list_bitmap_fill(const MaskArgs& a, const ReqMas
     }
 }
 
-// Which of the `slots` masks (one per head that shares this KV row) keep distance o.
+// LIST: which of the `slots` masks (one per head that shares this KV row) keep distance o.
 template <int SLOTS>
 __device__ __forceinline__ unsigned keep_bits(const MaskArgs& a, const ReqMask& m,
                                               const unsigned* bitmaps, int o) {
     constexpr unsigned ALL = (1u << SLOTS) - 1u;
     if (m.keep_all) return ALL;
-    if (a.mode == MODE_GRID) return grid_keep(m, a.stride, o) ? ALL : 0u;
     unsigned bits = 0;
 #pragma unroll
     for (int s = 0; s < SLOTS; ++s) {
@@ -132,14 +122,12 @@ __device__ __forceinline__ unsigned keep_bits(const MaskArgs& a, const ReqMask& 
     return bits;
 }
 
-// How the NT threads that build a list wait for each other: the whole block, or (in the persistent
-// kernel, where a loader warp runs beside them) a named barrier over the compute warps only.
+// How the threads that build a list wait for each other: a whole block, or one warp.
 struct BlockSync {
     __device__ static __forceinline__ void sync() { __syncthreads(); }
 };
-template <int NTHREADS>
-struct NamedSync {
-    __device__ static __forceinline__ void sync() { asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory"); }
+struct WarpSync {
+    __device__ static __forceinline__ void sync() { __syncwarp(); }
 };
 
 // Exclusive scan of one int per thread over NT threads (threadIdx.x < NT, NT a multiple of 32).
@@ -184,24 +172,46 @@ __device__ __forceinline__ int enumerate_kept(const MaskArgs& a, const ReqMask& 
         return m.prefix + m.n_win;
     }
     // Each thread owns a contiguous run of window candidates (ascending position = descending
-    // distance): count, scan, then emit.
+    // distance): count, scan, then emit.  The run is walked with the distance split as
+    // o = k * stride + r kept up to date incrementally, so the GRID test needs no division.
     const int per = (m.n_win + NT - 1) / NT;
     const int c0 = min((int)threadIdx.x * per, m.n_win), c1 = min(c0 + per, m.n_win);
-    // a sink that is still inside the window is kept whatever the mask says
-    auto bits_at = [&](int c) -> unsigned {
-        return (m.w_lo + c < m.sink_end) ? ALL : keep_bits<SLOTS>(a, m, bitmaps, m.T - c);
+    const bool grid = a.mode == MODE_GRID;
+    const int o_first = m.T - c0;
+    const int k_first = grid ? o_first / a.stride : 0;
+    const int r_first = grid ? o_first - k_first * a.stride : 0;
+    auto bits_at = [&](int c, int o, int k, int r) -> unsigned {
+        if (m.w_lo + c < m.sink_end) return ALL;        // a sink still inside the window is always kept
+        if (grid) {
+            if (o == m.T) return ALL;
+            const int d = min(r, a.stride - r);
+            if (d != m.dstar) return d < m.dstar ? ALL : 0u;
+            const int rank = (m.dstar == 0 || 2 * m.dstar == a.stride) ? k : 2 * k + (r == m.dstar ? 0 : 1);
+            return rank < m.need ? ALL : 0u;
+        }
+        return keep_bits<SLOTS>(a, m, bitmaps, o);
     };
     int cnt = 0;
-    for (int c = c0; c < c1; ++c) cnt += bits_at(c) != 0u;
+    {
+        int o = o_first, k = k_first, r = r_first;
+        for (int c = c0; c < c1; ++c) {
+            cnt += bits_at(c, o, k, r) != 0u;
+            --o;
+            if (--r < 0) { r = a.stride - 1; --k; }
+        }
+    }
     int total;
     int rank = m.prefix + block_excl_scan<NT, Sync>(cnt, total, s_warp);
     if (rank < r1 && rank + cnt > r0) {
+        int o = o_first, k = k_first, r = r_first;
         for (int c = c0; c < c1; ++c) {
-            const unsigned bits = bits_at(c);
+            const unsigned bits = bits_at(c, o, k, r);
             if (bits) {
                 if (rank >= r0 && rank < r1) sink(rank - r0, m.w_lo + c, bits);
                 ++rank;
             }
+            --o;
+            if (--r < 0) { r = a.stride - 1; --k; }
         }
     }
     return m.prefix + total;

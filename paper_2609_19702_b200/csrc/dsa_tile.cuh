@@ -50,8 +50,8 @@ struct RowList {
 };
 
 // Mask generator -> row list of split `split`.  Returns the number of rows written (0: nothing
-// kept in this split).  All NT compute threads call it.
-template <class C, class Sync>
+// kept in this split).  All NTHR threads that work on the item call it.
+template <class C, class Sync, int NTHR = NT>
 __device__ __forceinline__ int build_row_list(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split,
                                               const RowList& list, unsigned* bitmaps, int* s_warp) {
     const int tid = threadIdx.x;
@@ -59,32 +59,42 @@ __device__ __forceinline__ int build_row_list(const AttnArgs& a, const ReqMask& 
     if (m.keep_all && r0 >= m.prefix + m.n_win) return 0;
     if (a.mask.mode == MODE_LIST && !m.keep_all) {
         Sync::sync();                                     // bitmaps of the previous item are done with
-        for (int i = tid; i < C::SLOTS * a.mask.bitmap_words; i += NT) bitmaps[i] = 0u;
+        for (int i = tid; i < C::SLOTS * a.mask.bitmap_words; i += NTHR) bitmaps[i] = 0u;
         Sync::sync();
 #pragma unroll
         for (int s = 0; s < C::SLOTS; ++s) {
             const int h = kvh * C::G + s;
             const int mh = a.mask.mask_heads == 1 ? 0 : (a.mask.mask_heads == a.H_kv ? kvh : h);
             const int* trace = a.mask.skip_offsets + ((int64_t)b * a.mask.mask_heads + mh) * a.mask.trace_len;
-            list_bitmap_fill<NT>(a.mask, m, trace, bitmaps + s * a.mask.bitmap_words);
+            list_bitmap_fill<NTHR>(a.mask, m, trace, bitmaps + s * a.mask.bitmap_words);
         }
         Sync::sync();
     }
-    const int64_t head_off = (int64_t)kvh * a.stride_head;
-    const int total = enumerate_kept<NT, C::SLOTS, Sync>(a.mask, m, bitmaps, r0, r1, s_warp,
+    // Pass 1: the kept positions (nothing but integer work and shared-memory stores).
+    const int total = enumerate_kept<NTHR, C::SLOTS, Sync>(a.mask, m, bitmaps, r0, r1, s_warp,
         [&](int slot, int pos, unsigned bits) {
-            list.rowoff[slot] = token_offset(a, b, m.L_p, pos) + head_off;
+            list.rowoff[slot] = pos;
             if (C::SELECT) list.rowpos[slot] = pos;
             if (C::HEADMASK) list.hbits[slot] = (unsigned char)bits;
         });
-    return max(0, min(total - r0, a.chunk));
+    const int n_rows = max(0, min(total - r0, a.chunk));
+    Sync::sync();
+    // Pass 2: positions -> element offsets.  The block-table lookups of different rows are
+    // independent loads (neighbouring rows mostly hit the same table entries), so they overlap
+    // instead of queueing behind one another as they would inside the scan.
+    const int64_t head_off = (int64_t)kvh * a.stride_head;
+#pragma unroll 4
+    for (int i = tid; i < n_rows; i += NTHR)
+        list.rowoff[i] = token_offset(a, b, m.L_p, (int)list.rowoff[i]) + head_off;
+    return n_rows;
 }
 
 // Nothing kept in this split: lse = -inf (and out = 0 when this item owns the result).
-template <class C>
-__device__ __forceinline__ void write_empty_item(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split) {
+// Called by the NTHR threads that own the item; `tid` is the caller's index among them.
+template <class C, int NTHR = NT>
+__device__ __forceinline__ void write_empty_item(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split,
+                                                 int tid = threadIdx.x) {
     using T = typename C::T;
-    const int tid = threadIdx.x;
     if (a.n_split > 1) {
         if (tid < C::G) {
             const int64_t row = (int64_t)b * a.H_q + kvh * C::G + tid;
@@ -96,7 +106,7 @@ __device__ __forceinline__ void write_empty_item(const AttnArgs& a, const ReqMas
             }
         }
     } else {
-        for (int i = tid; i < C::G * C::D; i += NT)
+        for (int i = tid; i < C::G * C::D; i += NTHR)
             Elem<T>::store(a.out, ((int64_t)b * a.H_q + kvh * C::G) * C::D + i, 0.f);
         if (tid < C::G) a.lse[(int64_t)b * a.H_q + kvh * C::G + tid] = -INFINITY;
         if (C::SELECT && tid < C::G && m.sel_k >= 0)

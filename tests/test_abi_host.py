@@ -98,7 +98,8 @@ def test_plan_sizes(dsa):
     # sparse: prompt + N_att rows per kv head fit one block -> no split, one launch
     rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,
                                    max_prompt_len=200), _diag(dsa, window=512, n_att=208, grid_w=64))
-    assert rc == 0 and info.n_split == 1 and info.launches == 1 and info.grid_blocks == 256 * 32
+    assert rc == 0 and info.n_split == 1 and info.launches == 1
+    assert info.grid_blocks in (256 * 32, 256 * 16, 256 * 8)     # 1, 2 or 4 kv heads per block
     # dense on the same problem needs splits and the combine kernel
     rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360))
     assert rc == 0 and info.n_split * info.split_tokens >= 4360 and info.launches == 2
