@@ -37,7 +37,12 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch of the timed kernel from an ncu capture (see profiles/), keyed by the
 # workload string of the JSON line; None until a capture of that exact launch exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # ncu at batch 32: 209.38 MB read + 4.77 MB written per launch (profiles/dsa_attn_mma_kernel_...md);
+    # traffic grows in proportion to the batch, so a batch-256 launch moves 8 x that
+    "config5_paged_sweep B=256 Hq=32 Hkv=32 D=128 Lp=200 grid=64x64+1 paged16 sparse grid-mask window=512 n_att=208":
+        8 * 214_143_000,
+}
 
 
 def parse_args():
@@ -413,7 +418,8 @@ def run_ours(args):
                 "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(name),
                 "peak_kind": "of " + peak_kind, "algorithmic_bytes": abytes,
                 "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-                "kernel": "dsa_attn_kernel" + (" + dsa_combine_kernel" if plan.launches > 1 else "")}
+                "kernel": ("dsa_attn_mma_kernel" if plan.tensor_cores else "dsa_attn_kernel") +
+                          (" + dsa_combine_kernel" if plan.launches > 1 else "")}
 
     # ---- variants: dense and the other window, same library, same batch --------------------
     variants = {}
@@ -495,7 +501,8 @@ def run_ours(args):
                        "parallelism": "requests sharded over %d GPU(s), no collective" % world,
                        "plan": {"split_tokens": plan.split_tokens, "n_split": plan.n_split,
                                 "grid_blocks": plan.grid_blocks, "smem_bytes": plan.smem_bytes,
-                                "tile_tokens": plan.tile_tokens, "stages": plan.stages}},
+                                "tile_tokens": plan.tile_tokens, "stages": plan.stages,
+                                "tensor_cores": plan.tensor_cores, "work_items": plan.work_items}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }

@@ -173,7 +173,10 @@ typedef struct dsa_plan_info {
     int32_t grid_blocks;    /* thread blocks of the attention kernel                               */
     int32_t smem_bytes;     /* dynamic shared memory per block                                     */
     int32_t tile_tokens;    /* tokens per staged K/V tile                                          */
-    int32_t stages;         /* tiles in flight per block                                           */
+    int32_t stages;         /* tiles in flight per block (per warp for the tensor-core kernel)     */
+    int32_t tensor_cores;   /* 1: tensor-core kernel (bf16), one warp per work item;               */
+                            /* 0: CUDA-core kernel (fp32), one 128-thread block per work item      */
+    int32_t work_items;     /* (request, kv head, split) items                                     */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);
