@@ -255,6 +255,33 @@ def per_config_table(torch, dsa, synth, dev, peak):
     return rows
 
 
+def selection_overhead(torch, dsa, synth, dev):
+    """Cost of the fused phase-2 selection: config 5 at batch 256 with per-head LIST masks, every
+    request at a phase-2 position (N_att <= p < N_r), the sparse call with and without `select`."""
+    w = synth.workload(5, batch=256)
+    inputs = synth.make_inputs_device(w, dev)
+    rng = np.random.default_rng(synth.BASE_SEED + 5)
+    p = rng.integers(w.n_att, w.window, size=w.batch).astype(np.int32)
+    seq = torch.from_numpy(w.prompt_len + p).to(dev)
+    few = synth.random_valid_trace(rng, w.window, w.n_att, (8,))
+    trace = torch.from_numpy(np.ascontiguousarray(
+        few[rng.integers(0, 8, size=(w.batch, w.num_q_heads))])).to(dev)
+    prob = dsa.Problem(
+        q=inputs["q"], k_cache=inputs["k_cache"], v_cache=inputs["v_cache"], strides=inputs["strides"],
+        seq_len=seq, prompt_len=inputs["prompt_len"], num_kv_heads=w.num_kv_heads,
+        max_seq_len=inputs["max_seq_len"], max_prompt_len=w.prompt_len, block_table=inputs["block_table"],
+        block_size=inputs["block_size"], num_blocks=inputs["block_table"].numel())
+    out, lse = dsa.alloc_outputs(prob)
+    res = {"batch": w.batch, "window": w.window, "n_att": w.n_att, "mask": "per-head list"}
+    for name, sel in (("without_select", False), ("with_select", True)):
+        diag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=trace, select=sel)
+        ws = dsa.alloc_workspace(prob, diag)
+        secs, _ = time_calls(torch, lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws), 50, 5)
+        res[name + "_us"] = round(secs / 50 * 1e6, 2)
+    res["overhead_pct"] = round(100.0 * (res["with_select_us"] / res["without_select_us"] - 1.0), 2)
+    return res
+
+
 def decode_loop_bench(torch, dsa, synth, dev, n_layers=8):
     """Whole-image decode loop: 1024 image tokens after a 50-token prompt, batch 16, 32/32 heads,
     head_dim 128 -- the shape of the paper's Lumina-mGPT latency runs -- over `n_layers` layers,
@@ -452,16 +479,11 @@ def run_ours(args):
         h_bt = None if inputs["block_table"] is None else inputs["block_table"].cpu().pin_memory()
         h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
         h_lse = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+        e2e_ws = dsa.alloc_workspace(prob, diag)
 
         def e2e_step():
-            inputs["q"].copy_(h_q, non_blocking=True)
-            inputs["seq_len"].copy_(h_seq, non_blocking=True)
-            inputs["prompt_len"].copy_(h_pl, non_blocking=True)
-            if h_bt is not None:
-                inputs["block_table"].copy_(h_bt, non_blocking=True)
-            call()
-            h_out.copy_(out, non_blocking=True)
-            h_lse.copy_(lse, non_blocking=True)
+            # the C-ABI call with host buffers: H2D of the step's inputs, attention, D2H of the result
+            dsa.dsa_decode_attention_host_io(prob, diag, h_q, h_seq, h_pl, h_bt, out, lse, h_out, h_lse, e2e_ws)
             torch.cuda.current_stream().synchronize()      # the caller needs the result to go on
 
         esteps = min(args.steps, 100)
@@ -473,21 +495,22 @@ def run_ours(args):
         d2h = h_out.numel() * h_out.element_size() + h_lse.numel() * h_lse.element_size()
         e2e = {"value": round(world * w.batch * esteps / float(te.item()), 1), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": esteps,
-               "note": "per step: q, seq_len, prompt_len and block table from pinned host memory, "
-                       "out and lse back to pinned host memory, stream synchronised; the KV cache is "
-                       "decode state and stays resident in HBM"}
+               "note": "dsa_decode_attention_host_io per step: q, seq_len, prompt_len and block table from "
+                       "pinned host memory, out and lse back to pinned host memory, stream synchronised; "
+                       "the KV cache is decode state and stays resident in HBM"}
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload ------------------
     cpu = None
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
-    per_config = decode_loop = None
+    per_config = decode_loop = selection = None
     if args.all_configs and rank == 0 and world == 1:
         del inputs, prob, out, lse
         torch.cuda.empty_cache()
         per_config = per_config_table(torch, dsa, synth, dev, peak)
         decode_loop = decode_loop_bench(torch, dsa, synth, dev)
+        selection = selection_overhead(torch, dsa, synth, dev)
 
     if rank == 0:
         line = {
@@ -509,6 +532,7 @@ def run_ours(args):
         if per_config is not None:
             line["per_config"] = per_config
             line["decode_loop"] = decode_loop
+            line["selection_overhead"] = selection
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -211,6 +211,24 @@ DSA_API int32_t dsa_decode_attention_sparse(const dsa_problem *problem, const ds
                                     void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * One decode step's attention with the step's inputs and results in HOST memory (the call a
+ * serving loop makes when the scheduler lives on the CPU; the KV cache, which is decode state,
+ * stays on the device).  Not in the paper; it is the dense (diag == NULL) or sparse call above
+ * wrapped in the copies a step needs, all queued on `stream`:
+ *   host_q -> problem->q, host_seq_len -> problem->seq_len, host_prompt_len -> problem->prompt_len,
+ *   host_block_table -> problem->block_table (paged caches only; NULL otherwise),
+ *   attention into dev_out / dev_lse, then dev_out -> host_out, dev_lse -> host_lse.
+ * The device pointers inside `problem` are therefore WRITTEN by this call.  Host buffers should
+ * be pinned for the copies to be asynchronous; they must stay valid, and host_out / host_lse
+ * must not be read, until the stream has been synchronised by the caller.
+ */
+DSA_API int32_t dsa_decode_attention_host_io(const dsa_problem *problem, const dsa_diag_params *diag,
+                                             const void *host_q, const int32_t *host_seq_len,
+                                             const int32_t *host_prompt_len, const int32_t *host_block_table,
+                                             void *dev_out, float *dev_lse, void *host_out, float *host_lse,
+                                             void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Merge split-KV partial results (not in the paper; the exact identity that a softmax over a
  * union of key sets is the lse-weighted mix of the softmaxes over the parts):
  *   lse = ln sum_i e^{lse_i},  out = sum_i e^{lse_i - lse} out_i.

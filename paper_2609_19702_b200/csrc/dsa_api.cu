@@ -439,6 +439,39 @@ int32_t dsa_decode_attention_sparse(const dsa_problem* problem, const dsa_diag_p
     return run_attention(problem, diag, out, lse, workspace, workspace_bytes, stream);
 }
 
+int32_t dsa_decode_attention_host_io(const dsa_problem* problem, const dsa_diag_params* diag,
+                                     const void* host_q, const int32_t* host_seq_len,
+                                     const int32_t* host_prompt_len, const int32_t* host_block_table,
+                                     void* dev_out, float* dev_lse, void* host_out, float* host_lse,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+    const int32_t rc = check_problem(problem);
+    if (rc != DSA_OK) return rc;
+    if (problem->batch == 0) return DSA_OK;
+    if (!host_q || !host_seq_len || !host_prompt_len || !host_out || !host_lse || !dev_out || !dev_lse)
+        return DSA_ERR_INVALID_ARG;
+    if ((problem->block_table != nullptr) != (host_block_table != nullptr)) return DSA_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esize = problem->dtype == DSA_BF16 ? 2 : 4;
+    const size_t n_q = (size_t)problem->batch * problem->num_q_heads * problem->head_dim;
+    const size_t n_rows = (size_t)problem->batch * problem->num_q_heads;
+    cudaError_t e = cudaMemcpyAsync(const_cast<void*>(problem->q), host_q, n_q * esize, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(const_cast<int32_t*>(problem->seq_len), host_seq_len, (size_t)problem->batch * 4,
+                            cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(const_cast<int32_t*>(problem->prompt_len), host_prompt_len, (size_t)problem->batch * 4,
+                            cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && host_block_table)
+        e = cudaMemcpyAsync(const_cast<int32_t*>(problem->block_table), host_block_table,
+                            (size_t)problem->batch * problem->max_blocks * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int32_t rc2 = run_attention(problem, diag, dev_out, dev_lse, workspace, workspace_bytes, stream);
+    if (rc2 != DSA_OK) return rc2;
+    e = cudaMemcpyAsync(host_out, dev_out, n_q * esize, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(host_lse, dev_lse, n_rows * 4, cudaMemcpyDeviceToHost, st);
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+}
+
 int32_t dsa_combine_splits(const float* out_part, const float* lse_part, int32_t batch, int32_t num_q_heads,
                            int32_t head_dim, int32_t n_split, void* out, float* lse, int32_t out_dtype,
                            void* stream) {

@@ -200,3 +200,32 @@ def test_append_into_a_paged_linear_cache(dsa):
         expect[blk, seq[b] % 4] = k_new[b]
         assert torch.equal(vc[blk, seq[b] % 4].view(torch.int16), v_new[b].view(torch.int16))
     assert torch.equal(kc.view(torch.int16), expect.view(torch.int16))
+
+
+def test_host_io_call_matches_device_call(dsa):
+    w = synth.workload(5, batch=3)
+    inp = synth.make_inputs(w)
+    prob = dsa.problem_from_host(inp)
+    diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    for dg in (None, diag):
+        ref_out, ref_lse = dsa.alloc_outputs(prob)
+        ws = dsa.alloc_workspace(prob, dg)
+        if dg is None:
+            dsa.dsa_decode_attention_dense(prob, ref_out, ref_lse, ws)
+        else:
+            dsa.dsa_decode_attention_sparse(prob, dg, ref_out, ref_lse, ws)
+        torch.cuda.synchronize()
+        h_q = prob.q.cpu().pin_memory()
+        h_seq, h_pl = prob.seq_len.cpu().pin_memory(), prob.prompt_len.cpu().pin_memory()
+        h_bt = prob.block_table.cpu().pin_memory()
+        # scramble the device copies: the call must restore them from the host buffers
+        prob.q.zero_()
+        prob.seq_len.zero_()
+        prob.block_table.zero_()
+        out, lse = dsa.alloc_outputs(prob)
+        h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        h_lse = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+        dsa.dsa_decode_attention_host_io(prob, dg, h_q, h_seq, h_pl, h_bt, out, lse, h_out, h_lse, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(h_out.view(torch.int16), ref_out.cpu().view(torch.int16))
+        assert torch.equal(h_lse, ref_lse.cpu())
