@@ -1,0 +1,94 @@
+"""Randomised parity: many small problems with random shapes, layouts and mask parameters, the
+CUDA library against the oracle.  Seeds are fixed, so a failure reproduces."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as ora
+from paper_2609_19702_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _random_case(rng):
+    g = int(rng.choice([1, 2, 4, 8]))
+    hkv = int(rng.choice([1, 2, 3, 4, 6]))
+    d = int(rng.choice([64, 128]))
+    grid_w = int(rng.integers(1, 40))
+    extra = int(rng.integers(0, 2))
+    grid_h = int(rng.integers(1, max(2, 400 // (grid_w + extra))))
+    n_img = grid_h * (grid_w + extra)
+    n_r = int(rng.integers(1, min(n_img, 300) + 1))
+    n_att = int(rng.integers(1, n_r + 1))
+    l_p = int(rng.choice([0, 1, 5, 17, 64, 200]))
+    paged = bool(rng.integers(0, 2))
+    bs = int(rng.choice([1, 4, 16, 32]))
+    batch = int(rng.integers(1, 6))
+    return synth.Workload("fuzz", 0, batch, g * hkv, hkv, d, l_p, grid_h, grid_w, extra, n_r, n_att, 1, n_img,
+                          positional=bool(rng.integers(0, 2)), paged=paged, block_size=bs)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_problem(seed):
+    from paper_2609_19702_b200 import binding as dsa
+    rng = np.random.default_rng(9000 + seed)
+    w = _random_case(rng)
+    inp = synth.make_inputs(w, seed=500 + seed)
+    f32 = bool(rng.integers(0, 4) == 0)
+    split = int(rng.choice([0, 0, 16, 48, 130]))
+    prob = dsa.problem_from_host(inp, dtype=torch.float32 if f32 else torch.bfloat16, split_tokens=split)
+    n_sink = int(rng.choice([0, 0, 1, 4]))
+    hq, hkv = w.num_q_heads, w.num_kv_heads
+    mh = int(rng.choice(sorted({1, hkv, hq})))
+    trace = synth.random_valid_trace(rng, w.window, w.n_att, (w.batch, mh))
+    cases = [
+        (None, ora.MODE_DENSE, {}),
+        (dsa.Diag(dsa.DSA_MASK_WINDOW, w.window, n_sink=n_sink), ora.MODE_WINDOW, dict(n_r=w.window, n_sink=n_sink)),
+        (dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra, n_sink=n_sink), ora.MODE_GRID,
+         dict(n_r=w.window, n_att=w.n_att, stride=w.stride, n_sink=n_sink)),
+        (dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=torch.from_numpy(trace).cuda(), n_sink=n_sink),
+         ora.MODE_LIST, dict(n_r=w.window, n_att=w.n_att, trace=trace, n_sink=n_sink)),
+    ]
+    tag = "seed %d: %s f32=%s split=%d sinks=%d mh=%d" % (seed, w, f32, split, n_sink, mh)
+    for diag, mode, kw in cases:
+        ref = util.oracle_run(inp, mode, want_kept=True, **kw)
+        out, lse = dsa.alloc_outputs(prob)
+        out.fill_(float("nan"))
+        ws = dsa.alloc_workspace(prob, diag)
+        if diag is None:
+            dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+        else:
+            dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+        torch.cuda.synchronize()
+        util.assert_close(out, lse, ref, f32, "%s mode %d" % (tag, mode))
+        idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, inp["max_seq_len"])
+        util.assert_kept_equal(idx, cnt, ref, "%s mode %d" % (tag, mode))
+
+
+def test_long_single_sequence_many_splits():
+    # one request, 20 000 cached tokens, grouped heads: 20+ splits per kv head and a wide LIST window
+    from paper_2609_19702_b200 import binding as dsa
+    w = synth.Workload("long", 0, 1, 8, 2, 128, 300, 100, 197, 0, 4096, 1500, 19000, 19700)
+    inp = synth.make_inputs(w, seed=77)
+    prob = dsa.problem_from_host(inp)
+    assert dsa.dsa_query_plan(prob, None).n_split >= 20
+    rng = np.random.default_rng(3)
+    trace = synth.random_valid_trace(rng, w.window, w.n_att, (1, 8))
+    for diag, mode, kw in (
+            (None, ora.MODE_DENSE, {}),
+            (dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, 0), ora.MODE_GRID,
+             dict(n_r=w.window, n_att=w.n_att, stride=w.stride)),
+            (dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=torch.from_numpy(trace).cuda()),
+             ora.MODE_LIST, dict(n_r=w.window, n_att=w.n_att, trace=trace))):
+        ref = util.oracle_run(inp, mode, want_kept=True, **kw)
+        out, lse = dsa.alloc_outputs(prob)
+        ws = dsa.alloc_workspace(prob, diag)
+        if diag is None:
+            dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+        else:
+            dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+        torch.cuda.synchronize()
+        util.assert_close(out, lse, ref, what="long mode %d" % mode)
+        idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, inp["max_seq_len"])
+        util.assert_kept_equal(idx, cnt, ref, "long mode %d" % mode)
