@@ -327,18 +327,41 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
 }
 
+// `after_attention`: the combine follows the attention kernel of the same call.  It is then
+// launched with programmatic stream serialisation: its blocks may be scheduled while the last wave
+// of the attention kernel is still running (the attention kernels signal early with
+// griddepcontrol.launch_dependents) and wait inside the kernel (griddepcontrol.wait) until that
+// grid has completed and its writes are visible -- the launch latency of the second kernel hides
+// behind the first.
+template <typename T>
+cudaError_t launch_combine_t(const float* out_part, const float* lse_part, int64_t rows, int D, int n_split,
+                             void* out, float* lse, cudaStream_t st, const float* sel_val, const int* sel_off,
+                             const int* sel_k, int* trace, int trace_len, bool after_attention) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)rows);
+    cfg.blockDim = dim3((unsigned)D);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_attention ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, dsa_combine_kernel<T>, out_part, lse_part, D, n_split, out, lse, sel_val,
+                              sel_off, sel_k, trace, trace_len);
+}
+
 int32_t launch_combine(const float* out_part, const float* lse_part, int64_t rows, int D, int n_split,
                        void* out, float* lse, int dtype, cudaStream_t st, const float* sel_val = nullptr,
                        const int* sel_off = nullptr, const int* sel_k = nullptr, int* trace = nullptr,
-                       int trace_len = 0) {
+                       int trace_len = 0, bool after_attention = false) {
     if (rows == 0) return DSA_OK;
-    if (dtype == DSA_BF16)
-        dsa_combine_kernel<__nv_bfloat16><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse,
-                                                                      sel_val, sel_off, sel_k, trace, trace_len);
-    else
-        dsa_combine_kernel<float><<<(unsigned)rows, D, 0, st>>>(out_part, lse_part, D, n_split, out, lse,
-                                                              sel_val, sel_off, sel_k, trace, trace_len);
-    const cudaError_t e = cudaGetLastError();
+    const cudaError_t e =
+        dtype == DSA_BF16
+            ? launch_combine_t<__nv_bfloat16>(out_part, lse_part, rows, D, n_split, out, lse, st, sel_val, sel_off,
+                                              sel_k, trace, trace_len, after_attention)
+            : launch_combine_t<float>(out_part, lse_part, rows, D, n_split, out, lse, st, sel_val, sel_off, sel_k,
+                                      trace, trace_len, after_attention);
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
@@ -379,7 +402,7 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     if (pl.n_split > 1)
         return launch_combine(a.out_part, a.lse_part, (int64_t)p->batch * p->num_q_heads, p->head_dim,
                               pl.n_split, out, lse, p->dtype, st, a.sel_val_part, a.sel_off_part, a.sel_k,
-                              pl.select ? d->skip_offsets : nullptr, pl.select ? d->trace_len : 0);
+                              pl.select ? d->skip_offsets : nullptr, pl.select ? d->trace_len : 0, true);
     return DSA_OK;
 }
 

@@ -37,6 +37,9 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     using C = AttnCfg<T, D, G, TILE_N, STAGES, HEADMASK, SELECT>;
     constexpr int LPR = C::LPR, VEC = C::VEC;
 
+    // a combine kernel queued behind this grid may be scheduled from now on (it waits for this
+    // grid to finish before it reads anything)
+    asm volatile("griddepcontrol.launch_dependents;");
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_warp[NT / 32];
     unsigned char* pipe = smem;
@@ -105,6 +108,9 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
                                    const int* __restrict__ sel_off_part = nullptr,
                                    const int* __restrict__ sel_k = nullptr, int* trace = nullptr,
                                    int trace_len = 0) {
+    // launched behind an attention kernel with programmatic serialisation: wait for that grid
+    // and its writes (returns at once after an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t row = blockIdx.x;
     const float* lp = lse_part + row * n_split;
     float M = -INFINITY;
