@@ -35,6 +35,25 @@ int env_int(const char* name, int fallback) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Launch `kern` so that it may be scheduled before the kernel queued ahead of it on the stream has
+// finished (programmatic stream serialisation).  Every kernel launched this way starts with
+// griddepcontrol.wait, which holds it until that earlier grid has completed and its writes are
+// visible; after a kernel that never signals early this is an ordinary serialised launch.
+template <class Kern, class... Args>
+cudaError_t launch_pdl(Kern kern, unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 // The launch plan: how many kept rows one block takes, how many splits that makes.
 struct Plan {
     int mode;            // MODE_*
@@ -95,8 +114,7 @@ struct KernelPick {
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
         }
-        kern<<<(unsigned)grid, 32 * W, smem_bytes, st>>>(a);
-        return cudaGetLastError();
+        return launch_pdl(kern, (unsigned)grid, 32 * W, smem_bytes, st, a);
     }
     static cudaError_t launch_mma(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
@@ -120,8 +138,7 @@ struct KernelPick {
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
         }
-        kern<<<(unsigned)grid, NT, smem_bytes, st>>>(a);
-        return cudaGetLastError();
+        return launch_pdl(kern, (unsigned)grid, NT, smem_bytes, st, a);
     }
 };
 

@@ -37,9 +37,12 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     using C = AttnCfg<T, D, G, TILE_N, STAGES, HEADMASK, SELECT>;
     constexpr int LPR = C::LPR, VEC = C::VEC;
 
-    // a combine kernel queued behind this grid may be scheduled from now on (it waits for this
-    // grid to finish before it reads anything)
+    // Programmatic launch on both sides: a combine kernel queued behind this grid may be scheduled
+    // from now on (it waits for this grid to finish before it reads anything), and this grid may
+    // itself have been scheduled early behind the append kernel of the same decode step: wait for
+    // that kernel's writes (the new K/V rows, seq_len) before touching global memory.
     asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_warp[NT / 32];
     unsigned char* pipe = smem;
@@ -153,6 +156,9 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
 template <typename T>
 __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_new, const T* __restrict__ v_new,
                                      int D, int capacity, bool advance) {
+    // the attention kernel of this decode step may be scheduled behind this grid right away; it
+    // waits for this grid's writes before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
     const int S = a.seq_len[b];
     if (S < 0 || S >= capacity) return;                   // no room: the token is dropped

@@ -97,9 +97,12 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     constexpr unsigned FULL = 0xffffffffu;
     static_assert(W == 1 || (!HEADMASK && !SELECT), "a shared row list needs a head-independent mask");
 
-    // a combine kernel queued behind this grid may be scheduled from now on (it waits for this
-    // grid to finish before it reads anything)
+    // Programmatic launch on both sides: a combine kernel queued behind this grid may be scheduled
+    // from now on (it waits for this grid to finish before it reads anything), and this grid may
+    // itself have been scheduled early behind the append kernel of the same decode step: wait for
+    // that kernel's writes (the new K/V rows, seq_len) before touching global memory.
     asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_warp[W];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
