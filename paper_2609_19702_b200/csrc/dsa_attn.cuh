@@ -195,8 +195,9 @@ __global__ void __launch_bounds__(NT) dsa_kept_indices_kernel(const AttnArgs a, 
         __syncthreads();
     }
     int* dst = idx_out + (int64_t)blockIdx.x * max_kept;
-    const int total = enumerate_kept<NT, 1, BlockSync>(a.mask, m, bitmap, 0, max_kept, s_warp,
-                                            [&](int slot, int pos, unsigned) { dst[slot] = pos; });
+    auto write_pos = [&](int slot, int pos, unsigned) { dst[slot] = pos; };
+    enumerate_direct<NT, 1>(m, 0, max_kept, write_pos);
+    const int total = enumerate_scanned<NT, 1, BlockSync>(a.mask, m, bitmap, 0, max_kept, s_warp, write_pos);
     if (threadIdx.x == 0) count_out[blockIdx.x] = total;
 }
 

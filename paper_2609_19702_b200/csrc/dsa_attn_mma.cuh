@@ -118,19 +118,17 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     const int b = blockIdx.x / (hblocks * a.n_split);
 
     const ReqMask m = req_mask_setup(a.mask, a.seq_len[b], a.prompt_len[b], a.max_seq_len);
+    auto sync_builders = [&]() { if (W == 1) __syncwarp(); else __syncthreads(); };
     // W > 1: one list for all the block's heads, built without a head offset (kv head "0")
-    const int n_rows = W == 1 ? build_row_list<IC, WarpSync, 32>(a, m, b, kvh, split, list, bitmaps, s_warp)
-                              : build_row_list<IC, BlockSync, 32 * W>(a, m, b, 0, split, list, bitmaps, s_warp);
-    if (n_rows <= 0) { write_empty_item<IC, 32>(a, m, b, kvh, split, lane); return; }
-    if (W == 1) __syncwarp(); else __syncthreads();     // the last barrier: from here on warps run free
+    const int list_kvh = W == 1 ? kvh : 0;
     const int64_t head_bytes = W == 1 ? 0 : (int64_t)kvh * a.stride_head * 2;
-
-    // ---- staging: this warp's own ring of 16-key tiles ---------------------------------------
-    const int n_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
     const unsigned char* kbase = reinterpret_cast<const unsigned char*>(a.k);
     const unsigned char* vbase = reinterpret_cast<const unsigned char*>(a.v);
-    auto issue_tile = [&](int tile) {
-        if (tile < n_tiles) {
+
+    // ---- staging: this warp's own ring of 16-key tiles ---------------------------------------
+    // rows_ready: rows of the list that exist so far (tiles below it can be issued)
+    auto issue_tile = [&](int tile, int rows_ready) {
+        if (tile * MMA_KEYS < rows_ready) {
             unsigned char* ks = ring + (tile % STAGES) * C::SLOT_BYTES;
             unsigned char* vs = ks + C::TILE_BYTES;
 #pragma unroll
@@ -138,7 +136,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
                 const int idx = i * 32 + lane;
                 const int row = idx / C::CPR, c = idx % C::CPR;
                 const int r = tile * MMA_KEYS + row;
-                const bool valid = r < n_rows;
+                const bool valid = r < rows_ready;
                 const int64_t off = valid ? list.rowoff[r] * 2 + head_bytes + c * 16 : 0;
                 const int dst = row * C::ROW_BYTES + ((c ^ (row & 7)) * 16);       // swizzled chunk
                 cp_async16_w(ks + dst, kbase + off, valid);
@@ -147,8 +145,22 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
         }
         asm volatile("cp.async.commit_group;\n" ::);
     };
-#pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) issue_tile(s);
+
+    // Phase A of the row list: the rows that need no scan (prompt, old sinks, unmasked window).
+    // The first tiles of the ring are issued from them right away, so that the memory stream is
+    // already running while phase B (mask bitmaps, window scan, block-table lookups) is computed.
+    const int n_direct = W == 1 ? build_rows_direct<IC, 32>(a, m, b, list_kvh, split, list)
+                                : build_rows_direct<IC, 32 * W>(a, m, b, list_kvh, split, list);
+    sync_builders();
+    const int early = min(STAGES - 1, n_direct / MMA_KEYS);          // whole tiles inside phase A
+    for (int s = 0; s < early; ++s) issue_tile(s, n_direct);
+    const int n_rows = W == 1
+        ? build_rows_scanned<IC, WarpSync, 32>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct)
+        : build_rows_scanned<IC, BlockSync, 32 * W>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct);
+    if (n_rows <= 0) { write_empty_item<IC, 32>(a, m, b, kvh, split, lane); return; }
+    sync_builders();                                   // the last barrier: from here on warps run free
+    const int n_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
+    for (int s = early; s < STAGES - 1; ++s) issue_tile(s, n_rows);
 
     // ---- Q^T as B operand: head = lane / 4, dims 2*(lane%4)+{0,1} (+8) of every 16-dim step ----
     const int hq = lane >> 2;                 // head column this thread feeds
@@ -184,7 +196,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     for (int tile = 0; tile < n_tiles; ++tile) {
         asm volatile("cp.async.wait_group %0;\n" ::"n"(STAGES - 2));
         __syncwarp();                                   // tile landed for every lane; tile-1 fully consumed
-        issue_tile(tile + STAGES - 1);
+        issue_tile(tile + STAGES - 1, n_rows);
         const unsigned char* ks = ring + (tile % STAGES) * C::SLOT_BYTES;
         const unsigned char* vs = ks + C::TILE_BYTES;
 

@@ -154,23 +154,31 @@ __device__ __forceinline__ int block_excl_scan(int v, int& total, int* s_warp /*
     return base + incl - v;
 }
 
-// Enumerate the kept positions with union rank in [r0, r1), calling
+// The kept positions are enumerated in two parts, both calling
 //   sink(rank - r0, cache position, head bits)
-// for each, and return the total number of kept positions (union over the SLOTS masks).
-// All NT threads must call it (it synchronises through Sync).
-template <int NT, int SLOTS, class Sync, class Sink>
-__device__ __forceinline__ int enumerate_kept(const MaskArgs& a, const ReqMask& m,
-                                              const unsigned* bitmaps, int r0, int r1,
-                                              int* s_warp, Sink sink) {
+// for the kept positions with union rank in [r0, r1).
+//
+// Part 1, "direct": the ranks whose position follows from the rank alone -- the prompt, the sinks
+// that have left the window, and the whole window when nothing is skipped.  No scan, no barrier.
+// Returns how many ranks of [r0, r1) it covered (they are the first ones of the split).
+template <int NT, int SLOTS, class Sink>
+__device__ __forceinline__ int enumerate_direct(const ReqMask& m, int r0, int r1, Sink sink) {
     constexpr unsigned ALL = (1u << SLOTS) - 1u;
-    // the prompt (always attended in full) and the sinks that have left the window
-    for (int r = max(r0, 0) + (int)threadIdx.x; r < min(r1, m.prefix); r += NT) sink(r - r0, r, ALL);
-    if (m.keep_all) {
-        // contiguous window: rank prefix + c  <->  position w_lo + c
-        const int lo = max(r0, m.prefix), hi = min(r1, m.prefix + m.n_win);
-        for (int r = lo + (int)threadIdx.x; r < hi; r += NT) sink(r - r0, m.w_lo + (r - m.prefix), ALL);
-        return m.prefix + m.n_win;
-    }
+    const int direct_end = m.keep_all ? m.prefix + m.n_win : m.prefix;
+    const int hi = min(r1, direct_end);
+    for (int r = r0 + (int)threadIdx.x; r < hi; r += NT)
+        sink(r - r0, r < m.prefix ? r : m.w_lo + (r - m.prefix), ALL);
+    return max(0, hi - r0);
+}
+
+// Part 2, "scanned": the window under a mask.  All NT threads must call it (it synchronises through
+// Sync).  Returns the total number of kept positions of the request (direct ones included).
+template <int NT, int SLOTS, class Sync, class Sink>
+__device__ __forceinline__ int enumerate_scanned(const MaskArgs& a, const ReqMask& m,
+                                                 const unsigned* bitmaps, int r0, int r1,
+                                                 int* s_warp, Sink sink) {
+    constexpr unsigned ALL = (1u << SLOTS) - 1u;
+    if (m.keep_all) return m.prefix + m.n_win;
     // Each thread owns a contiguous run of window candidates (ascending position = descending
     // distance): count, scan, then emit.  The run is walked with the distance split as
     // o = k * stride + r kept up to date incrementally, so the GRID test needs no division.

@@ -49,16 +49,37 @@ struct RowList {
     }
 };
 
-// Mask generator -> row list of split `split`.  Returns the number of rows written (0: nothing
-// kept in this split).  All NTHR threads that work on the item call it.
+// Mask generator -> row list of split `split`, in two phases so that a kernel can start streaming
+// the rows of phase A while phase B is still being computed.  All NTHR threads that work on the
+// item call both.
+//
+// Phase A: the rows whose position needs no scan (prompt, old sinks, an unmasked window).  Writes
+// their final element offsets and returns how many there are; they are rows [0, n) of the list.
+// The caller synchronises before anyone reads them.
+template <class C, int NTHR = NT>
+__device__ __forceinline__ int build_rows_direct(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split,
+                                                 const RowList& list) {
+    const int r0 = split * a.chunk, r1 = r0 + a.chunk;
+    const int64_t head_off = (int64_t)kvh * a.stride_head;
+    return enumerate_direct<NTHR, C::SLOTS>(m, r0, r1, [&](int slot, int pos, unsigned bits) {
+        list.rowoff[slot] = token_offset(a, b, m.L_p, pos) + head_off;
+        if (C::SELECT) list.rowpos[slot] = pos;
+        if (C::HEADMASK) list.hbits[slot] = (unsigned char)bits;
+    });
+}
+
+// Phase B: the window under a mask (rows [n_direct, n_rows) of the list).  Returns n_rows, the
+// number of rows of the whole split.  The caller synchronises before anyone reads the new rows.
 template <class C, class Sync, int NTHR = NT>
-__device__ __forceinline__ int build_row_list(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split,
-                                              const RowList& list, unsigned* bitmaps, int* s_warp) {
+__device__ __forceinline__ int build_rows_scanned(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split,
+                                                  const RowList& list, unsigned* bitmaps, int* s_warp,
+                                                  int n_direct) {
     const int tid = threadIdx.x;
     const int r0 = split * a.chunk, r1 = r0 + a.chunk;
-    if (m.keep_all && r0 >= m.prefix + m.n_win) return 0;
-    if (a.mask.mode == MODE_LIST && !m.keep_all) {
-        Sync::sync();                                     // bitmaps of the previous item are done with
+    if (m.keep_all) return n_direct;
+    if (r0 >= m.prefix + m.n_win) return n_direct;            // beyond anything a mask could keep
+    if (a.mask.mode == MODE_LIST) {
+        Sync::sync();                                     // bitmaps of a previous use are done with
         for (int i = tid; i < C::SLOTS * a.mask.bitmap_words; i += NTHR) bitmaps[i] = 0u;
         Sync::sync();
 #pragma unroll
@@ -71,7 +92,7 @@ __device__ __forceinline__ int build_row_list(const AttnArgs& a, const ReqMask& 
         Sync::sync();
     }
     // Pass 1: the kept positions (nothing but integer work and shared-memory stores).
-    const int total = enumerate_kept<NTHR, C::SLOTS, Sync>(a.mask, m, bitmaps, r0, r1, s_warp,
+    const int total = enumerate_scanned<NTHR, C::SLOTS, Sync>(a.mask, m, bitmaps, r0, r1, s_warp,
         [&](int slot, int pos, unsigned bits) {
             list.rowoff[slot] = pos;
             if (C::SELECT) list.rowpos[slot] = pos;
@@ -84,9 +105,17 @@ __device__ __forceinline__ int build_row_list(const AttnArgs& a, const ReqMask& 
     // instead of queueing behind one another as they would inside the scan.
     const int64_t head_off = (int64_t)kvh * a.stride_head;
 #pragma unroll 4
-    for (int i = tid; i < n_rows; i += NTHR)
+    for (int i = n_direct + tid; i < n_rows; i += NTHR)
         list.rowoff[i] = token_offset(a, b, m.L_p, (int)list.rowoff[i]) + head_off;
     return n_rows;
+}
+
+// Both phases back to back.
+template <class C, class Sync, int NTHR = NT>
+__device__ __forceinline__ int build_row_list(const AttnArgs& a, const ReqMask& m, int b, int kvh, int split,
+                                              const RowList& list, unsigned* bitmaps, int* s_warp) {
+    const int n_direct = build_rows_direct<C, NTHR>(a, m, b, kvh, split, list);
+    return build_rows_scanned<C, Sync, NTHR>(a, m, b, kvh, split, list, bitmaps, s_warp, n_direct);
 }
 
 // Nothing kept in this split: lse = -inf (and out = 0 when this item owns the result).
