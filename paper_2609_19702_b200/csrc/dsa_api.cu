@@ -97,7 +97,6 @@ struct KernelPick {
     static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, kMmaStages, HM, SEL, W>::smem_bytes(chunk, bw); }
     static size_t smem_mma(int w, int chunk, int bw) {
         if constexpr (!HM && !SEL) {
-            if (w == 4) return smem_mma_w<4>(chunk, bw);
             if (w == 2) return smem_mma_w<2>(chunk, bw);
         }
         return smem_mma_w<1>(chunk, bw);
@@ -119,7 +118,6 @@ struct KernelPick {
     static cudaError_t launch_mma(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
             if constexpr (!HM && !SEL) {
-                if (w == 4) return launch_mma_w<4>(a, items / 4, smem_bytes, st);
                 if (w == 2) return launch_mma_w<2>(a, items / 2, smem_bytes, st);
             }
             return launch_mma_w<1>(a, items, smem_bytes, st);
@@ -267,8 +265,8 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         pl->tile = MMA_KEYS;
         pl->stages = kMmaStages;
         const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
-        if (shared_mask) pl->mma_warps = p->num_kv_heads % 4 == 0 ? 4 : (p->num_kv_heads % 2 == 0 ? 2 : 1);
-        pl->mma_warps = std::min(pl->mma_warps, 2);     // measured: 2 heads per block beat 1 and 4
+        // two kv heads per block (measured: 2 beats 1 and 4) when the row list can be shared
+        if (shared_mask && p->num_kv_heads % 2 == 0) pl->mma_warps = 2;
     }
 
     int chunk;
