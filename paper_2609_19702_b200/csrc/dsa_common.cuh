@@ -31,7 +31,6 @@ struct AttnArgs {
     int chunk;                   // kept rows per split (multiple of the tile, <= MAX_CHUNK)
     int n_split;
     int n_items;                 // B * H_kv * n_split work items
-    int ring_slots;              // persistent kernel: tiles in its shared-memory ring
     void* out;                   // n_split == 1: [B, H_q, D] in T
     float* lse;                  //               [B, H_q]
     float* out_part;             // n_split > 1:  [B, H_q, n_split, D]
@@ -40,7 +39,6 @@ struct AttnArgs {
     float* sel_val_part;         // [B, H_q, n_split] lowest logit (base 2) among this split's candidates
     int* sel_off_part;           // [B, H_q, n_split] its distance behind the query, -1 if none
     int* sel_k;                  // [B, H_q] trace entry to write, -1 if this request selects nothing
-    int* error_flag;             // persistent kernel: set if a bounded wait ran out
 };
 
 // Where token `pos` (logical cache position) of request b lives, as an element offset of its kv
