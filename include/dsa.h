@@ -21,6 +21,9 @@
  *     kernels clamp them into range instead, so bad values give wrong numbers, not faults.
  *   - Return value: DSA_OK or a negative dsa_status.  After DSA_ERR_CUDA the CUDA error code is
  *     available from dsa_last_cuda_error().
+ *   - The first launch of each kernel variant on a device also configures it (a one-time
+ *     attribute call); make the first call of a given shape outside any stream capture.  After
+ *     that the attention, combine and append calls can be captured into CUDA graphs.
  *   - There is no CPU path: without a CUDA device every compute call fails with DSA_ERR_CUDA.
  *
  * Positions.  For request b, prompt_len[b] = L_p tokens of prompt come first in the cache and

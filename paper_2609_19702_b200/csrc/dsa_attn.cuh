@@ -10,15 +10,6 @@
 
 namespace dsa {
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, bool valid) {
-    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
-    const int src_size = valid ? 16 : 0;     // 0: nothing is read, the 16 bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_size));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
-
 template <typename T, int D, int G, int TILE_N, int STAGES, bool HEADMASK, bool SELECT = false>
 struct AttnCfg : ItemCfg<T, D, G, TILE_N, HEADMASK, SELECT> {
     using Base = ItemCfg<T, D, G, TILE_N, HEADMASK, SELECT>;

@@ -55,12 +55,6 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
-__device__ __forceinline__ void cp_async16_w(void* smem_dst, const void* gmem_src, bool valid) {
-    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
-    const int src_size = valid ? 16 : 0;     // 0: nothing is read, the 16 bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_size));
-}
-
 template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W = 1>
 struct MmaCfg {
     using T = __nv_bfloat16;
@@ -139,11 +133,11 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
                 const bool valid = r < rows_ready;
                 const int64_t off = valid ? list.rowoff[r] * 2 + head_bytes + c * 16 : 0;
                 const int dst = row * C::ROW_BYTES + ((c ^ (row & 7)) * 16);       // swizzled chunk
-                cp_async16_w(ks + dst, kbase + off, valid);
-                cp_async16_w(vs + dst, vbase + off, valid);
+                cp_async16(ks + dst, kbase + off, valid);
+                cp_async16(vs + dst, vbase + off, valid);
             }
         }
-        asm volatile("cp.async.commit_group;\n" ::);
+        cp_async_commit();
     };
 
     // Phase A of the row list: the rows that need no scan (prompt, old sinks, unmasked window).
@@ -194,7 +188,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     const int lm_chk_v = (lane >> 3) & 1;
 
     for (int tile = 0; tile < n_tiles; ++tile) {
-        asm volatile("cp.async.wait_group %0;\n" ::"n"(STAGES - 2));
+        cp_async_wait<STAGES - 2>();
         __syncwarp();                                   // tile landed for every lane; tile-1 fully consumed
         issue_tile(tile + STAGES - 1, n_rows);
         const unsigned char* ks = ring + (tile % STAGES) * C::SLOT_BYTES;
@@ -256,7 +250,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
             mma_bf16_16816(o[mt], af, pb0, pb1);
         }
     }
-    asm volatile("cp.async.wait_group 0;\n" ::);
+    cp_async_wait<0>();
 
     // ---- finish: sums over the key lanes, normalise, write ------------------------------------
 #pragma unroll

@@ -241,3 +241,15 @@ def test_skipped_rows_are_never_read(dsa):
     diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
     out, lse = _run_gpu(dsa, prob, diag)
     util.assert_close(out, lse, ref, what="poisoned")
+
+
+def test_kept_index_export_truncates_but_counts_everything(dsa):
+    w = synth.workload(1)
+    inp = synth.make_inputs(w)
+    prob = dsa.problem_from_host(inp)
+    diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    full_idx, full_cnt = dsa.dsa_debug_kept_indices(prob, diag, inp["max_seq_len"])
+    idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, 20)
+    torch.cuda.synchronize()
+    assert torch.equal(cnt, full_cnt) and int(cnt.max()) > 20
+    assert torch.equal(idx[:, :, :20], full_idx[:, :, :20])
