@@ -355,7 +355,7 @@ cudaError_t launch_combine_t(const float* out_part, const float* lse_part, int64
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)rows);
     cfg.blockDim = dim3((unsigned)D);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = (size_t)n_split * sizeof(float);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -514,6 +514,7 @@ int32_t dsa_combine_splits(const float* out_part, const float* lse_part, int32_t
                            int32_t head_dim, int32_t n_split, void* out, float* lse, int32_t out_dtype,
                            void* stream) {
     if (batch < 0 || num_q_heads < 1 || head_dim < 1 || head_dim > 1024 || n_split < 1) return DSA_ERR_INVALID_ARG;
+    if (n_split > 8192) return DSA_ERR_UNSUPPORTED;              // weights live in 32 KB of shared memory
     if (out_dtype != DSA_BF16 && out_dtype != DSA_F32) return DSA_ERR_UNSUPPORTED;
     if (batch == 0) return DSA_OK;
     if (!out_part || !lse_part || !out) return DSA_ERR_INVALID_ARG;

@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
 }
 
 // ---- split combine: one block per (request, query head), one thread per output element -------
+// Launch with n_split * 4 bytes of dynamic shared memory.
 // With sel_k != nullptr it also finishes Algorithm 1's selection: the lowest candidate logit over
 // the splits (equal logits: the oldest key, i.e. the largest distance) becomes trace entry sel_k.
 template <typename T>
@@ -105,26 +106,54 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
     // launched behind an attention kernel with programmatic serialisation: wait for that grid
     // and its writes (returns at once after an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Dynamic shared memory: n_split weights.  The lse values are loaded once, in parallel, the
+    // maximum and the sum are block reductions, and the weighted sum then reads the partial
+    // outputs with independent loads: no chain of dependent global loads as long as n_split.
+    extern __shared__ float s_w[];
+    __shared__ float s_red[32];
     const int64_t row = blockIdx.x;
     const float* lp = lse_part + row * n_split;
-    float M = -INFINITY;
-    for (int i = 0; i < n_split; ++i) M = fmaxf(M, lp[i]);
-    float den = 0.f;
-    if (M != -INFINITY)
-        for (int i = 0; i < n_split; ++i) den += lp[i] == -INFINITY ? 0.f : expf(lp[i] - M);
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = (nthr + 31) >> 5;
+    auto block_reduce = [&](float v, bool is_max) -> float {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            const float o = __shfl_xor_sync(0xffffffffu, v, off);
+            v = is_max ? fmaxf(v, o) : v + o;
+        }
+        __syncthreads();                                 // s_red free again
+        if (lane == 0) s_red[warp] = v;
+        __syncthreads();
+        float r = s_red[0];
+        for (int w = 1; w < nwarp; ++w) r = is_max ? fmaxf(r, s_red[w]) : r + s_red[w];
+        return r;
+    };
+    float mx = -INFINITY;
+    for (int i = tid; i < n_split; i += nthr) {
+        const float v = lp[i];
+        s_w[i] = v;
+        mx = fmaxf(mx, v);
+    }
+    const float M = block_reduce(mx, true);
+    float part = 0.f;
+    for (int i = tid; i < n_split; i += nthr) {          // each thread revisits the entries it wrote
+        const float v = s_w[i];
+        const float w = (v == -INFINITY || M == -INFINITY) ? 0.f : expf(v - M);
+        s_w[i] = w;
+        part += w;
+    }
+    const float den = block_reduce(part, false);         // (its barriers also publish s_w)
     const float inv = den > 0.f ? 1.f / den : 0.f;
-    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    for (int d = tid; d < D; d += nthr) {
         float num = 0.f;
-        if (den > 0.f) {
-            for (int i = 0; i < n_split; ++i) {
-                const float li = lp[i];
-                if (li == -INFINITY) continue;            // empty part: its out_i is not read
-                num = fmaf(expf(li - M), out_part[(row * n_split + i) * D + d], num);
-            }
+        const float* op = out_part + row * n_split * D + d;
+#pragma unroll 4
+        for (int i = 0; i < n_split; ++i) {
+            const float w = s_w[i];
+            if (w != 0.f) num = fmaf(w, op[(int64_t)i * D], num);   // an empty part's out_i is not read
         }
         Elem<T>::store(out, row * D + d, num * inv);
     }
-    if (threadIdx.x == 0 && lse) lse[row] = den > 0.f ? M + logf(den) : -INFINITY;
+    if (tid == 0 && lse) lse[row] = den > 0.f ? M + logf(den) : -INFINITY;
     if (threadIdx.x == 0 && sel_k != nullptr) {
         const int k = sel_k[row];
         if (k >= 0) {
