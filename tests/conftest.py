@@ -12,6 +12,15 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (runs the sm_100a library)")
 
 
+def pytest_sessionstart(session):
+    # Build the CUDA library (nvcc cross-compiles, no GPU needed) and the C oracle if their sources
+    # are newer than the binaries; both are no-ops when up to date.
+    from paper_2609_19702_b200 import build as cuda_build
+    from oracle import oracle as ora
+    cuda_build.build()
+    ora.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
