@@ -4,7 +4,6 @@
 
 #include <cmath>
 #include <cstdio>
-
 #include <cstdlib>
 
 #include "dsa_attn.cuh"
