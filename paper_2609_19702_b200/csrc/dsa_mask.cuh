@@ -199,11 +199,17 @@ __device__ __forceinline__ int enumerate_scanned(const MaskArgs& a, const ReqMas
         }
         return keep_bits<SLOTS>(a, m, bitmaps, o);
     };
+    // Pass 1 counts and, for a single mask and a run of at most 32 candidates, remembers the
+    // verdicts in a bit mask so that pass 2 only has to walk the set bits.
+    const bool remember = SLOTS == 1 && per <= 32;
+    unsigned verdicts = 0u;
     int cnt = 0;
     {
         int o = o_first, k = k_first, r = r_first;
         for (int c = c0; c < c1; ++c) {
-            cnt += bits_at(c, o, k, r) != 0u;
+            const bool keep = bits_at(c, o, k, r) != 0u;
+            cnt += keep;
+            if (remember && keep) verdicts |= 1u << (c - c0);
             --o;
             if (--r < 0) { r = a.stride - 1; --k; }
         }
@@ -211,15 +217,24 @@ __device__ __forceinline__ int enumerate_scanned(const MaskArgs& a, const ReqMas
     int total;
     int rank = m.prefix + block_excl_scan<NT, Sync>(cnt, total, s_warp);
     if (rank < r1 && rank + cnt > r0) {
-        int o = o_first, k = k_first, r = r_first;
-        for (int c = c0; c < c1; ++c) {
-            const unsigned bits = bits_at(c, o, k, r);
-            if (bits) {
-                if (rank >= r0 && rank < r1) sink(rank - r0, m.w_lo + c, bits);
+        if (remember) {
+            while (verdicts) {
+                const int j = __ffs(verdicts) - 1;
+                verdicts &= verdicts - 1u;
+                if (rank >= r0 && rank < r1) sink(rank - r0, m.w_lo + c0 + j, ALL);
                 ++rank;
             }
-            --o;
-            if (--r < 0) { r = a.stride - 1; --k; }
+        } else {
+            int o = o_first, k = k_first, r = r_first;
+            for (int c = c0; c < c1; ++c) {
+                const unsigned bits = bits_at(c, o, k, r);
+                if (bits) {
+                    if (rank >= r0 && rank < r1) sink(rank - r0, m.w_lo + c, bits);
+                    ++rank;
+                }
+                --o;
+                if (--r < 0) { r = a.stride - 1; --k; }
+            }
         }
     }
     return m.prefix + total;
