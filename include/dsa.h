@@ -232,6 +232,26 @@ DSA_API int32_t dsa_decode_attention_host_io(const dsa_problem *problem, const d
                                              void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same step as dsa_decode_attention_host_io, with the large transfers folded into the
+ * kernels (not in the paper): the attention kernels read q from, and write out / lse to, the
+ * caller's PINNED host buffers directly over the bus (mapped, zero-copy), so no separate q upload
+ * precedes the attention and no download follows it.  What every head of a request re-reads
+ * (host_seq_len, host_prompt_len, host_block_table) is still copied into the device arrays named
+ * in `problem`, which are therefore WRITTEN.  problem->q is scratch: when the plan splits the
+ * keys of one (request, kv head) over several work items, q is first copied there so that it
+ * crosses the bus once; otherwise it is left untouched.
+ * host_q, host_out and host_lse must be page-locked host memory that the device can address
+ * (cudaHostAlloc / cudaHostRegister; checked with cudaPointerGetAttributes before anything is
+ * queued: DSA_ERR_INVALID_ARG otherwise), host_q and host_out 16-byte aligned.  They must stay valid, and
+ * host_out / host_lse must not be read, until the caller has synchronised the stream.
+ */
+DSA_API int32_t dsa_decode_attention_host_mapped(const dsa_problem *problem, const dsa_diag_params *diag,
+                                                 const void *host_q, const int32_t *host_seq_len,
+                                                 const int32_t *host_prompt_len, const int32_t *host_block_table,
+                                                 void *host_out, float *host_lse,
+                                                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Merge split-KV partial results (not in the paper; the exact identity that a softmax over a
  * union of key sets is the lse-weighted mix of the softmaxes over the parts):
  *   lse = ln sum_i e^{lse_i},  out = sum_i e^{lse_i - lse} out_i.

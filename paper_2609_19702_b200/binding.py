@@ -23,7 +23,8 @@ DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
 EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_workspace_size",
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
            "dsa_combine_splits", "dsa_debug_kept_indices",
-           "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io"]
+           "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
+           "dsa_decode_attention_host_mapped"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -80,6 +81,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
     lib.dsa_decode_attention_host_io.restype = i32
     lib.dsa_decode_attention_host_io.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.dsa_decode_attention_host_mapped.restype = i32
+    lib.dsa_decode_attention_host_mapped.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_append_kv.restype = i32
     lib.dsa_append_kv.argtypes = [vp, vp, vp, i32, vp]
     lib.dsa_debug_kept_indices.restype = i32
@@ -282,6 +285,28 @@ def dsa_decode_attention_host_io(problem: Problem, diag: Optional[Diag], host_q:
                                              _dptr(host_prompt_len), _dptr(host_block_table), _dptr(dev_out),
                                              _dptr(dev_lse), _dptr(host_out), _dptr(host_lse), _dptr(workspace),
                                              ws_n, _stream(stream)))
+
+
+def dsa_decode_attention_host_mapped(problem: Problem, diag: Optional[Diag], host_q: torch.Tensor,
+                                     host_seq_len: torch.Tensor, host_prompt_len: torch.Tensor,
+                                     host_block_table: Optional[torch.Tensor], host_out: torch.Tensor,
+                                     host_lse: torch.Tensor, workspace: Optional[torch.Tensor] = None,
+                                     stream: Optional[torch.cuda.Stream] = None) -> None:
+    """One decode step whose kernels read ``host_q`` from and write ``host_out`` / ``host_lse`` to
+    pinned host tensors directly; lengths and block table are copied into the device tensors of
+    ``problem`` (and ``problem.q`` may be used as scratch).  Raises DsaError (invalid argument) for
+    host tensors that are not pinned.  Asynchronous: synchronise the stream before reading the
+    results."""
+    for t in (host_q, host_seq_len, host_prompt_len, host_out, host_lse):
+        assert not t.is_cuda and t.is_contiguous()
+    p = problem.c_struct()
+    d = diag.c_struct() if diag is not None else None
+    ws_n = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check("dsa_decode_attention_host_mapped",
+           _lib.dsa_decode_attention_host_mapped(_ref(p), _ref(d), _dptr(host_q), _dptr(host_seq_len),
+                                                 _dptr(host_prompt_len), _dptr(host_block_table),
+                                                 _dptr(host_out), _dptr(host_lse), _dptr(workspace),
+                                                 ws_n, _stream(stream)))
 
 
 def dsa_combine_splits(out_part: torch.Tensor, lse_part: torch.Tensor, out: torch.Tensor,

@@ -509,6 +509,56 @@ int32_t dsa_decode_attention_host_io(const dsa_problem* problem, const dsa_diag_
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
+// The address under which the device reaches a page-locked host buffer; nullptr when `host` is
+// not such a buffer (pageable, device or unknown memory).
+static void* mapped_alias(const void* host) {
+    cudaPointerAttributes at = {};
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
+int32_t dsa_decode_attention_host_mapped(const dsa_problem* problem, const dsa_diag_params* diag,
+                                         const void* host_q, const int32_t* host_seq_len,
+                                         const int32_t* host_prompt_len, const int32_t* host_block_table,
+                                         void* host_out, float* host_lse, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+    Plan pl;
+    const int32_t rc = make_plan(problem, diag, &pl);
+    if (rc != DSA_OK) return rc;
+    if (problem->batch == 0) return DSA_OK;
+    if (!host_q || !host_seq_len || !host_prompt_len || !host_out || !host_lse) return DSA_ERR_INVALID_ARG;
+    if ((problem->block_table != nullptr) != (host_block_table != nullptr)) return DSA_ERR_INVALID_ARG;
+    void* q_dev = mapped_alias(host_q);
+    void* out_dev = mapped_alias(host_out);
+    float* lse_dev = reinterpret_cast<float*>(mapped_alias(host_lse));
+    if (!q_dev || !out_dev || !lse_dev) return DSA_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esize = problem->dtype == DSA_BF16 ? 2 : 4;
+    cudaError_t e = cudaMemcpyAsync(const_cast<int32_t*>(problem->seq_len), host_seq_len,
+                                    (size_t)problem->batch * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(const_cast<int32_t*>(problem->prompt_len), host_prompt_len, (size_t)problem->batch * 4,
+                            cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && host_block_table)
+        e = cudaMemcpyAsync(const_cast<int32_t*>(problem->block_table), host_block_table,
+                            (size_t)problem->batch * problem->max_blocks * 4, cudaMemcpyHostToDevice, st);
+    dsa_problem sub = *problem;
+    if (pl.n_split > 1) {
+        // every split of a (request, kv head) reads q: bring it over once
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(const_cast<void*>(problem->q), host_q,
+                                (size_t)problem->batch * problem->num_q_heads * problem->head_dim * esize,
+                                cudaMemcpyHostToDevice, st);
+    } else {
+        sub.q = q_dev;
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    return run_attention(&sub, diag, out_dev, lse_dev, workspace, workspace_bytes, stream);
+}
+
 int32_t dsa_combine_splits(const float* out_part, const float* lse_part, int32_t batch, int32_t num_q_heads,
                            int32_t head_dim, int32_t n_split, void* out, float* lse, int32_t out_dtype,
                            void* stream) {
