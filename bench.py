@@ -38,10 +38,10 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch of the timed kernel from an ncu capture (see profiles/), keyed by the
 # workload string of the JSON line; None until a capture of that exact launch exists.
 NCU_TRAFFIC_BYTES = {
-    # ncu at batch 32: 209.38 MB read + 4.77 MB written per launch (profiles/dsa_attn_mma_kernel_...md);
+    # ncu at batch 32: 209.39 MB read + 3.81 MB written per launch (profiles/dsa_attn_mma_kernel_...md);
     # traffic grows in proportion to the batch, so a batch-256 launch moves 8 x that
     "config5_paged_sweep B=256 Hq=32 Hkv=32 D=128 Lp=200 grid=64x64+1 paged16 sparse grid-mask window=512 n_att=208":
-        8 * 214_143_000,
+        8 * 213_193_600,
 }
 
 
