@@ -276,6 +276,35 @@ DSA_API int32_t dsa_append_kv(const dsa_problem *problem, const void *k_new, con
                               int32_t advance, void *stream);
 
 /*
+ * One decode step of one layer in a single launch (plus the combine when the plan splits):
+ * dsa_append_kv followed by the dense (diag == NULL) or sparse attention call, fused.  Not a
+ * method of its own: Algorithm 1's "K.append(K_t)" and "Attn(Q_t, K_p + K[idx], ...)" of one
+ * step, issued together.
+ *   seq_len[b] counts the tokens ALREADY cached, without the token being decoded, and is not
+ *   modified: a model's layers share one seq_len array, which the caller advances once per token
+ *   after its last layer (dsa_advance_seq_len).
+ *   k_new, v_new: device [B, H_kv, D] in problem->dtype, 16-byte aligned.  The rows of request b
+ *   are written to logical position seq_len[b] of the cache and the request attends over
+ *   seq_len[b] + 1 tokens, the mask taking p = seq_len[b] + 1 - prompt_len[b].  A request whose
+ *   seq_len is already max_seq_len has no room: its token is dropped and it attends over what
+ *   is cached, exactly as dsa_append_kv followed by attention would do.
+ * For bf16 the attention kernel itself reads the current token's rows from k_new / v_new and
+ * stores them to the cache; for float32 the rows are stored by a launch of their own first.
+ * Everything else (outputs, workspace, plan, fused selection, bounded caches) as for the
+ * attention calls.
+ */
+DSA_API int32_t dsa_decode_step(const dsa_problem *problem, const dsa_diag_params *diag,
+                                const void *k_new, const void *v_new, void *out, float *lse,
+                                void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * seq_len[b] += 1 for every request below `max_seq_len` (device array of `batch` int32), queued on
+ * `stream`: the once-per-token counterpart of dsa_decode_step, so that a captured token step
+ * (every layer's dsa_decode_step, then this) can be replayed without the host touching seq_len.
+ */
+DSA_API int32_t dsa_advance_seq_len(int32_t *seq_len, int32_t batch, int32_t max_seq_len, void *stream);
+
+/*
  * The kept cache positions, produced by the same device code that the sparse attention kernel
  * uses to decide which rows to read (Algorithm 1: K_p, then window - skip_idx as positions).
  * Positions are LOGICAL (before any ring mapping).

@@ -24,7 +24,7 @@ EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_works
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
            "dsa_combine_splits", "dsa_debug_kept_indices",
            "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
-           "dsa_decode_attention_host_mapped"]
+           "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -81,6 +81,10 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
     lib.dsa_decode_attention_host_io.restype = i32
     lib.dsa_decode_attention_host_io.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.dsa_decode_step.restype = i32
+    lib.dsa_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.dsa_advance_seq_len.restype = i32
+    lib.dsa_advance_seq_len.argtypes = [vp, i32, i32, vp]
     lib.dsa_decode_attention_host_mapped.restype = i32
     lib.dsa_decode_attention_host_mapped.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_append_kv.restype = i32
@@ -329,6 +333,31 @@ def dsa_append_kv(problem: Problem, k_new: torch.Tensor, v_new: torch.Tensor, ad
     p = problem.c_struct()
     _check("dsa_append_kv", _lib.dsa_append_kv(_ref(p), _dptr(k_new), _dptr(v_new), 1 if advance else 0,
                                                _stream(stream)))
+
+
+def dsa_decode_step(problem: Problem, diag: Optional[Diag], k_new: torch.Tensor, v_new: torch.Tensor,
+                    out: torch.Tensor, lse: torch.Tensor, workspace: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Append + attention of one decode step in one call: ``problem.seq_len`` counts the tokens
+    already cached (it is not advanced), ``k_new`` / ``v_new`` [B, H_kv, D] are the current token."""
+    b, _, d = problem.q.shape
+    for t in (k_new, v_new):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == problem.q.dtype
+        assert tuple(t.shape) == (b, problem.num_kv_heads, d)
+    p = problem.c_struct()
+    dg = diag.c_struct() if diag is not None else None
+    ws_n = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check("dsa_decode_step",
+           _lib.dsa_decode_step(_ref(p), _ref(dg), _dptr(k_new), _dptr(v_new), _dptr(out), _dptr(lse),
+                                _dptr(workspace), ws_n, _stream(stream)))
+
+
+def dsa_advance_seq_len(seq_len: torch.Tensor, max_seq_len: int,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """seq_len[b] += 1 on the device for every request below ``max_seq_len``."""
+    assert seq_len.is_cuda and seq_len.dtype == torch.int32 and seq_len.is_contiguous()
+    _check("dsa_advance_seq_len",
+           _lib.dsa_advance_seq_len(_dptr(seq_len), seq_len.numel(), int(max_seq_len), _stream(stream)))
 
 
 def dsa_debug_kept_indices(problem: Problem, diag: Optional[Diag], max_kept: int,

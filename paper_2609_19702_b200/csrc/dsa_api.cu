@@ -100,9 +100,9 @@ struct KernelPick {
         }
         return smem_mma_w<1>(chunk, bw);
     }
-    template <int W>
+    template <int W, bool APPEND>
     static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W>;
+        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND>;
         static bool configured[kMaxDevices] = {};
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -114,15 +114,22 @@ struct KernelPick {
         }
         return launch_pdl(kern, (unsigned)grid, 32 * W, smem_bytes, st, a);
     }
-    static cudaError_t launch_mma(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
+    // `append`: the fused decode step (the kernel reads the current token from a.k_new / a.v_new)
+    template <bool APPEND>
+    static cudaError_t launch_mma_a(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
             if constexpr (!HM && !SEL) {
-                if (w == 2) return launch_mma_w<2>(a, items / 2, smem_bytes, st);
+                if (w == 2) return launch_mma_w<2, APPEND>(a, items / 2, smem_bytes, st);
             }
-            return launch_mma_w<1>(a, items, smem_bytes, st);
+            return launch_mma_w<1, APPEND>(a, items, smem_bytes, st);
         } else {
             return cudaErrorInvalidValue;
         }
+    }
+    static cudaError_t launch_mma(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st,
+                                  bool append) {
+        return append ? launch_mma_a<true>(w, a, items, smem_bytes, st)
+                      : launch_mma_a<false>(w, a, items, smem_bytes, st);
     }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
         auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
@@ -339,6 +346,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->n_items = (int)pl.grid;
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
+    a->step_append = 0; a->k_new = nullptr; a->v_new = nullptr;
 }
 
 // `after_attention`: the combine follows the attention kernel of the same call.  It is then
@@ -379,13 +387,21 @@ int32_t launch_combine(const float* out_part, const float* lse_part, int64_t row
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
+int32_t launch_append(const dsa_problem* problem, const void* k_new, const void* v_new, bool advance,
+                      cudaStream_t st);
+
+// k_new / v_new non-NULL: the fused decode step -- seq_len counts the tokens already cached, the
+// token being decoded is appended by this call and attended to as well.
 int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out, float* lse,
-                      void* workspace, size_t workspace_bytes, void* stream) {
+                      void* workspace, size_t workspace_bytes, void* stream, const void* k_new = nullptr,
+                      const void* v_new = nullptr) {
     Plan pl;
     int32_t rc = make_plan(p, d, &pl);
     if (rc != DSA_OK) return rc;
     if (p->batch == 0) return DSA_OK;
     if (!out || !lse || !aligned16(out)) return DSA_ERR_INVALID_ARG;
+    const bool step = k_new != nullptr;
+    if (step && (!v_new || !aligned16(k_new) || !aligned16(v_new))) return DSA_ERR_INVALID_ARG;
     if (pl.ws_total > 0) {
         if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return DSA_ERR_INVALID_ARG;
         if (workspace_bytes < pl.ws_total) return DSA_ERR_WORKSPACE_TOO_SMALL;
@@ -405,10 +421,21 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
         a.out = out; a.lse = lse;
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (step) {
+        a.step_append = 1;
+        if (pl.mma) {
+            a.k_new = k_new; a.v_new = v_new;             // read and stored by the attention kernel itself
+        } else {
+            // CUDA-core kernel: the rows go to the cache in a launch of their own first
+            rc = launch_append(p, k_new, v_new, false, st);
+            if (rc != DSA_OK) return rc;
+        }
+    }
     cudaError_t err = cudaSuccess;
     rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, pl.select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
-        err = pl.mma ? P::launch_mma(pl.mma_warps, a, pl.grid, pl.smem, st) : P::launch(a, pl.grid, pl.smem, st);
+        err = pl.mma ? P::launch_mma(pl.mma_warps, a, pl.grid, pl.smem, st, step && pl.mma)
+                     : P::launch(a, pl.grid, pl.smem, st);
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;
@@ -418,6 +445,27 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
                               pl.n_split, out, lse, p->dtype, st, a.sel_val_part, a.sel_off_part, a.sel_k,
                               pl.select ? d->skip_offsets : nullptr, pl.select ? d->trace_len : 0, true);
     return DSA_OK;
+}
+
+int32_t launch_append(const dsa_problem* problem, const void* k_new, const void* v_new, bool advance,
+                      cudaStream_t st) {
+    Plan pl = {};
+    pl.mode = MODE_WINDOW;
+    pl.chunk = 0; pl.n_split = 1;
+    AttnArgs a;
+    fill_args(problem, nullptr, pl, &a);
+    const unsigned grid = (unsigned)problem->batch;
+    const int cap = problem->max_seq_len;
+    if (problem->dtype == DSA_BF16)
+        dsa_append_kv_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_new),
+                                                               reinterpret_cast<const __nv_bfloat16*>(v_new),
+                                                               problem->head_dim, cap, advance);
+    else
+        dsa_append_kv_kernel<float><<<grid, 256, 0, st>>>(a, reinterpret_cast<const float*>(k_new),
+                                                        reinterpret_cast<const float*>(v_new), problem->head_dim, cap,
+                                                        advance);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
 }  // namespace
@@ -577,22 +625,21 @@ int32_t dsa_append_kv(const dsa_problem* problem, const void* k_new, const void*
     if (rc != DSA_OK) return rc;
     if (problem->batch == 0) return DSA_OK;
     if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return DSA_ERR_INVALID_ARG;
-    Plan pl = {};
-    pl.mode = MODE_WINDOW;
-    pl.chunk = 0; pl.n_split = 1;
-    AttnArgs a;
-    fill_args(problem, nullptr, pl, &a);
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const unsigned grid = (unsigned)problem->batch;
-    const int cap = problem->max_seq_len;
-    if (problem->dtype == DSA_BF16)
-        dsa_append_kv_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_new),
-                                                               reinterpret_cast<const __nv_bfloat16*>(v_new),
-                                                               problem->head_dim, cap, advance != 0);
-    else
-        dsa_append_kv_kernel<float><<<grid, 256, 0, st>>>(a, reinterpret_cast<const float*>(k_new),
-                                                        reinterpret_cast<const float*>(v_new), problem->head_dim, cap,
-                                                        advance != 0);
+    return launch_append(problem, k_new, v_new, advance != 0, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int32_t dsa_decode_step(const dsa_problem* problem, const dsa_diag_params* diag, const void* k_new,
+                        const void* v_new, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+    if (!k_new || !v_new) return DSA_ERR_INVALID_ARG;
+    return run_attention(problem, diag, out, lse, workspace, workspace_bytes, stream, k_new, v_new);
+}
+
+int32_t dsa_advance_seq_len(int32_t* seq_len, int32_t batch, int32_t max_seq_len, void* stream) {
+    if (batch < 0 || max_seq_len < 0 || (batch > 0 && !seq_len)) return DSA_ERR_INVALID_ARG;
+    if (batch == 0) return DSA_OK;
+    dsa_advance_seq_len_kernel<<<(unsigned)((batch + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        seq_len, batch, max_seq_len);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }

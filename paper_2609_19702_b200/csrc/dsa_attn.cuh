@@ -47,7 +47,8 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     const int split = (blockIdx.x / a.H_kv) % a.n_split;
     const int b = blockIdx.x / (a.H_kv * a.n_split);
 
-    const ReqMask m = req_mask_setup(a.mask, a.seq_len[b], a.prompt_len[b], a.max_seq_len);
+    bool has_new;                                         // (the rows were appended by an earlier kernel)
+    const ReqMask m = req_mask_setup(a.mask, step_seq_len(a, b, has_new), a.prompt_len[b], a.max_seq_len);
     const int n_rows = build_row_list<C, BlockSync>(a, m, b, kvh, split, list, bitmaps, s_warp);
     if (n_rows <= 0) { write_empty_item<C>(a, m, b, kvh, split); return; }
     __syncthreads();
@@ -199,6 +200,12 @@ __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_n
     if (advance && threadIdx.x == 0) a.seq_len_rw[b] = S + 1;
 }
 
+// ---- seq_len[b] += 1 (not beyond the limit): once per decode step, after the last layer's fused step
+__global__ void dsa_advance_seq_len_kernel(int* seq_len, int batch, int limit) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch && seq_len[b] >= 0 && seq_len[b] < limit) seq_len[b] += 1;
+}
+
 // ---- debug export of the kept positions: one block per (request, mask head) ------------------
 __global__ void __launch_bounds__(NT) dsa_kept_indices_kernel(const AttnArgs a, int* idx_out, int* count_out,
                                                               int max_kept) {
@@ -206,7 +213,8 @@ __global__ void __launch_bounds__(NT) dsa_kept_indices_kernel(const AttnArgs a, 
     __shared__ int s_warp[NT / 32];
     const int mheads = a.mask.mode == MODE_LIST ? a.mask.mask_heads : 1;
     const int mh = blockIdx.x % mheads, b = blockIdx.x / mheads;
-    const ReqMask m = req_mask_setup(a.mask, a.seq_len[b], a.prompt_len[b], a.max_seq_len);
+    bool has_new;                                         // (the rows were appended by an earlier kernel)
+    const ReqMask m = req_mask_setup(a.mask, step_seq_len(a, b, has_new), a.prompt_len[b], a.max_seq_len);
     if (a.mask.mode == MODE_LIST && !m.keep_all) {
         for (int i = threadIdx.x; i < a.mask.bitmap_words; i += NT) bitmap[i] = 0u;
         __syncthreads();

@@ -83,7 +83,11 @@ struct MmaItemCfg {
     static constexpr int SLOTS = HEADMASK ? G : 1;
 };
 
-template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W>
+// APPEND: fused decode step.  The token being decoded is not in the cache yet: its K/V rows are
+// read from k_new / v_new wherever the row list names its position, and the warps of split 0
+// write them to the cache (nobody reads that slot in this launch: with a bounded cache it belonged
+// to a token that has left the window).
+template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false>
 __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) {
     using C = MmaCfg<D, G, STAGES, HEADMASK, SELECT, W>;
     using IC = MmaItemCfg<D, G, HEADMASK, SELECT>;
@@ -111,13 +115,32 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     const int split = (blockIdx.x / hblocks) % a.n_split;
     const int b = blockIdx.x / (hblocks * a.n_split);
 
-    const ReqMask m = req_mask_setup(a.mask, a.seq_len[b], a.prompt_len[b], a.max_seq_len);
+    bool has_new = false;
+    const int S_step = APPEND ? step_seq_len(a, b, has_new) : a.seq_len[b];
+    const ReqMask m = req_mask_setup(a.mask, S_step, a.prompt_len[b], a.max_seq_len);
     auto sync_builders = [&]() { if (W == 1) __syncwarp(); else __syncthreads(); };
     // W > 1: one list for all the block's heads, built without a head offset (kv head "0")
     const int list_kvh = W == 1 ? kvh : 0;
     const int64_t head_bytes = W == 1 ? 0 : (int64_t)kvh * a.stride_head * 2;
     const unsigned char* kbase = reinterpret_cast<const unsigned char*>(a.k);
     const unsigned char* vbase = reinterpret_cast<const unsigned char*>(a.v);
+    // fused step: where the current token's rows come from and where they go (kv head 0)
+    const unsigned char* knew_row = nullptr;
+    const unsigned char* vnew_row = nullptr;
+    int64_t off_new = 0;
+    int new_r = -1;                                       // its row in this item's list, once known
+    uint4 new_chunk = make_uint4(0u, 0u, 0u, 0u);
+    const bool store_new = APPEND && has_new && split == 0 && lane < 2 * C::CPR;
+    if (APPEND && has_new) {
+        const int64_t row_bytes = ((int64_t)b * a.H_kv + kvh) * C::ROW_BYTES;
+        knew_row = reinterpret_cast<const unsigned char*>(a.k_new) + row_bytes;
+        vnew_row = reinterpret_cast<const unsigned char*>(a.v_new) + row_bytes;
+        off_new = token_offset(a, b, m.L_p, m.S - 1);
+        if (store_new) {                                  // lanes [0, CPR): K chunks, [CPR, 2 CPR): V chunks
+            const unsigned char* src = lane < C::CPR ? knew_row + lane * 16 : vnew_row + (lane - C::CPR) * 16;
+            new_chunk = *reinterpret_cast<const uint4*>(src);
+        }
+    }
 
     // ---- staging: this warp's own ring of 16-key tiles ---------------------------------------
     // rows_ready: rows of the list that exist so far (tiles below it can be issued)
@@ -133,8 +156,13 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
                 const bool valid = r < rows_ready;
                 const int64_t off = valid ? list.rowoff[r] * 2 + head_bytes + c * 16 : 0;
                 const int dst = row * C::ROW_BYTES + ((c ^ (row & 7)) * 16);       // swizzled chunk
-                cp_async16(ks + dst, kbase + off, valid);
-                cp_async16(vs + dst, vbase + off, valid);
+                if (APPEND && r == new_r) {
+                    cp_async16(ks + dst, knew_row + c * 16, valid);
+                    cp_async16(vs + dst, vnew_row + c * 16, valid);
+                } else {
+                    cp_async16(ks + dst, kbase + off, valid);
+                    cp_async16(vs + dst, vbase + off, valid);
+                }
             }
         }
         cp_async_commit();
@@ -146,13 +174,22 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     const int n_direct = W == 1 ? build_rows_direct<IC, 32>(a, m, b, list_kvh, split, list)
                                 : build_rows_direct<IC, 32 * W>(a, m, b, list_kvh, split, list);
     sync_builders();
-    const int early = min(STAGES - 1, n_direct / MMA_KEYS);          // whole tiles inside phase A
+    // whole tiles inside phase A (fused step: never the newest row, which may not be in the cache)
+    const int early = min(STAGES - 1, (n_direct - (APPEND ? 1 : 0)) / MMA_KEYS);
     for (int s = 0; s < early; ++s) issue_tile(s, n_direct);
     const int n_rows = W == 1
         ? build_rows_scanned<IC, WarpSync, 32>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct)
         : build_rows_scanned<IC, BlockSync, 32 * W>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct);
+    if (store_new) {
+        unsigned char* base = const_cast<unsigned char*>(lane < C::CPR ? kbase : vbase);
+        const int c = lane < C::CPR ? lane : lane - C::CPR;
+        *reinterpret_cast<uint4*>(base + (off_new + (int64_t)kvh * a.stride_head) * 2 + c * 16) = new_chunk;
+    }
     if (n_rows <= 0) { write_empty_item<IC, 32>(a, m, b, kvh, split, lane); return; }
     sync_builders();                                   // the last barrier: from here on warps run free
+    // kept positions ascend, so the token being decoded can only be this item's last row
+    if (APPEND && has_new && list.rowoff[n_rows - 1] == off_new + (int64_t)list_kvh * a.stride_head)
+        new_r = n_rows - 1;
     const int n_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
     for (int s = early; s < STAGES - 1; ++s) issue_tile(s, n_rows);
 

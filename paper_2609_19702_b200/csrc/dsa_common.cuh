@@ -39,7 +39,20 @@ struct AttnArgs {
     float* sel_val_part;         // [B, H_q, n_split] lowest logit (base 2) among this split's candidates
     int* sel_off_part;           // [B, H_q, n_split] its distance behind the query, -1 if none
     int* sel_k;                  // [B, H_q] trace entry to write, -1 if this request selects nothing
+    // fused decode step: the cache holds seq_len[b] tokens and the call appends the token being
+    // decoded itself (logical position seq_len[b]) before attending over seq_len[b] + 1 tokens
+    int step_append;             // 0: seq_len counts the current token, nothing is appended
+    const void* k_new;           // [B, H_kv, D] rows of the current token; NULL: already in the cache
+    const void* v_new;
 };
+
+// Number of tokens request b attends over.  In a fused decode step that is one more than the
+// cache holds, unless the request is full (the token is then dropped, as by the append call).
+__device__ __forceinline__ int step_seq_len(const AttnArgs& a, int b, bool& has_new) {
+    const int S = a.seq_len[b];
+    has_new = a.step_append != 0 && S >= 0 && S < a.max_seq_len;
+    return has_new ? S + 1 : S;
+}
 
 // Where token `pos` (logical cache position) of request b lives, as an element offset of its kv
 // head 0.  With a bounded cache (ring_size > 0) the prompt and the first ring_sinks decode tokens
