@@ -282,14 +282,17 @@ def selection_overhead(torch, dsa, synth, dev):
     return res
 
 
-def decode_loop_bench(torch, dsa, synth, dev, n_layers=8):
-    """Whole-image decode loop: 1024 image tokens after a 50-token prompt, batch 16, 32/32 heads,
-    head_dim 128 -- the shape of the paper's Lumina-mGPT latency runs -- over `n_layers` layers,
-    each with its own KV cache (together larger than the L2).  Every step appends the new token's
-    K/V and attends, layer after layer; the step is captured once as a CUDA graph and replayed
-    1024 times.  Sparse: bounded ring cache, window 512, N_att 52 (95 % sparsity), grid mask.
-    Dense: full linear cache."""
-    b, h, d, l_p, grid = 16, 32, 128, 50, 32
+def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
+                      modes=("dense", "sparse", "sparse_select", "dense_two_calls", "sparse_two_calls")):
+    """Whole-image decode loop: 1024 image tokens after a 50-token prompt, `batch` requests (16: the
+    shape of the paper's Lumina-mGPT latency runs), 32/32 heads, head_dim 128, over `n_layers`
+    layers, each with its own KV cache (together larger than the L2).  Every step appends the new
+    token's K/V and attends, layer after layer: one fused dsa_decode_step per layer, the layers
+    sharing one seq_len array that is advanced once per token ("_two_calls" modes: dsa_append_kv +
+    attention per layer instead).  The step is captured once as a CUDA graph and replayed 1024
+    times.  Sparse: bounded ring cache, window 512, N_att 52 (95 % sparsity), grid mask.  Dense:
+    full linear cache."""
+    b, h, d, l_p, grid = batch, 32, 128, 50, 32
     steps = grid * grid
     s_max = l_p + steps
     row = h * d
@@ -298,35 +301,45 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8):
     res = {"batch": b, "heads": h, "head_dim": d, "prompt_len": l_p, "image_tokens": steps, "layers": n_layers}
     # "sparse": grid-derived diagonals (no selection work); "sparse_select": the paper's own method,
     # per-head list masks grown step by step by the fused phase-2 selection (argmin) in the call
-    for mode in ("dense", "sparse", "sparse_select"):
-        ring = 0 if mode == "dense" else 512
+    # "_two_calls": dsa_append_kv + attention per layer (each layer advancing its own seq_len);
+    # otherwise the fused dsa_decode_step per layer and one dsa_advance_seq_len per token
+    for mode in modes:
+        fused = not mode.endswith("_two_calls")
+        kind = mode.replace("_two_calls", "")
+        ring = 0 if kind == "dense" else 512
         cap = l_p + ring if ring else s_max
-        diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 52, grid, 0) if mode == "sparse" else None
+        diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 52, grid, 0) if kind == "sparse" else None
         q = torch.randn((b, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         k_new, v_new = q.clone(), q.clone()
+        shared_seq = torch.full((b,), l_p, dtype=torch.int32, device=dev)
         layers = []
         for _ in range(n_layers):
             kc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
             vc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
-            seq = torch.full((b,), l_p, dtype=torch.int32, device=dev)
+            seq = shared_seq if fused else torch.full((b,), l_p, dtype=torch.int32, device=dev)
             pl = torch.full((b,), l_p, dtype=torch.int32, device=dev)
             prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d),
                                seq_len=seq, prompt_len=pl, num_kv_heads=h, max_seq_len=s_max,
                                max_prompt_len=l_p, ring_size=ring)
             out, lse = dsa.alloc_outputs(prob)
             ldiag = diag
-            if mode == "sparse_select":
+            if kind == "sparse_select":
                 trace = torch.zeros((b, h, 512 - 52), dtype=torch.int32, device=dev)
                 ldiag = dsa.Diag(dsa.DSA_MASK_LIST, 512, 52, skip_offsets=trace, select=True)
             layers.append((prob, out, lse, dsa.alloc_workspace(prob, ldiag), ldiag))
 
         def step():
             for prob, out, lse, ws, ldiag in layers:
+                if fused:
+                    dsa.dsa_decode_step(prob, ldiag, k_new, v_new, out, lse, ws)
+                    continue
                 dsa.dsa_append_kv(prob, k_new, v_new, advance=True)
                 if ldiag is None:
                     dsa.dsa_decode_attention_dense(prob, out, lse, ws)
                 else:
                     dsa.dsa_decode_attention_sparse(prob, ldiag, out, lse, ws)
+            if fused:
+                dsa.dsa_advance_seq_len(shared_seq, s_max)
 
         def reset(value):
             for prob, _, _, _, _ in layers:
@@ -365,11 +378,13 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8):
         res[mode] = {"ms_per_image": round(best, 3), "us_per_step": round(best / steps * 1e3, 2),
                      "us_per_layer_step": round(best / steps / n_layers * 1e3, 2),
                      "us_last_step": round(last / reps * 1e3, 2), "cache_GB": round(cache_gb, 3),
-                     "n_split": plan.n_split, "launches_per_layer_step": plan.launches + 1}
+                     "n_split": plan.n_split,
+                     "launches_per_layer_step": plan.launches + (0 if fused else 1)}
         del layers, graph
         torch.cuda.empty_cache()
-    res["speedup_per_image_with_selection"] = round(
-        res["dense"]["ms_per_image"] / res["sparse_select"]["ms_per_image"], 3)
+    if "sparse_select" in res:
+        res["speedup_per_image_with_selection"] = round(
+            res["dense"]["ms_per_image"] / res["sparse_select"]["ms_per_image"], 3)
     res["speedup_per_image"] = round(res["dense"]["ms_per_image"] / res["sparse"]["ms_per_image"], 3)
     res["speedup_last_step"] = round(res["dense"]["us_last_step"] / res["sparse"]["us_last_step"], 3)
     res["cache_ratio"] = round(res["dense"]["cache_GB"] / res["sparse"]["cache_GB"], 3)
@@ -521,12 +536,15 @@ def run_ours(args):
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
-    per_config = decode_loop = selection = None
+    per_config = decode_loop = decode_loop_large = selection = None
     if args.all_configs and rank == 0 and world == 1:
         del inputs, prob, out, lse
         torch.cuda.empty_cache()
         per_config = per_config_table(torch, dsa, synth, dev, peak)
         decode_loop = decode_loop_bench(torch, dsa, synth, dev)
+        # the same loop at a batch where a B200 step is bandwidth-bound rather than latency-bound
+        decode_loop_large = decode_loop_bench(torch, dsa, synth, dev, batch=128,
+                                              modes=("dense", "sparse", "sparse_select"))
         selection = selection_overhead(torch, dsa, synth, dev)
 
     if rank == 0:
@@ -549,6 +567,7 @@ def run_ours(args):
         if per_config is not None:
             line["per_config"] = per_config
             line["decode_loop"] = decode_loop
+            line["decode_loop_batch128"] = decode_loop_large
             line["selection_overhead"] = selection
         print(json.dumps(line))
     if dist is not None:

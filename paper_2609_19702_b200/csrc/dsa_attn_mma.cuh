@@ -115,9 +115,24 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     const int split = (blockIdx.x / hblocks) % a.n_split;
     const int b = blockIdx.x / (hblocks * a.n_split);
 
+    const int seq_raw = a.seq_len[b], prompt_raw = a.prompt_len[b];
+    // ---- Q^T as B operand: head = lane / 4, dims 2*(lane%4)+{0,1} (+8) of every 16-dim step ----
+    // Loaded first, used last: the loads depend on nothing but the work item, so their latency
+    // hides behind the mask set-up and the row list (columns beyond the group are zeroed at use).
+    const int hq = lane >> 2;                 // head column this thread feeds
+    const int qd = (lane & 3) * 2;
+    unsigned qb[C::KSTEPS][2];
+    {
+        const T* qrow = reinterpret_cast<const T*>(a.q) + ((int64_t)b * a.H_q + kvh * G + (hq < G ? hq : 0)) * D;
+#pragma unroll
+        for (int kk = 0; kk < C::KSTEPS; ++kk) {
+            qb[kk][0] = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd);
+            qb[kk][1] = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd + 8);
+        }
+    }
     bool has_new = false;
-    const int S_step = APPEND ? step_seq_len(a, b, has_new) : a.seq_len[b];
-    const ReqMask m = req_mask_setup(a.mask, S_step, a.prompt_len[b], a.max_seq_len);
+    const int S_step = APPEND ? step_seq_len(a, seq_raw, has_new) : seq_raw;
+    const ReqMask m = req_mask_setup(a.mask, S_step, prompt_raw, a.max_seq_len);
     auto sync_builders = [&]() { if (W == 1) __syncwarp(); else __syncthreads(); };
     // W > 1: one list for all the block's heads, built without a head offset (kv head "0")
     const int list_kvh = W == 1 ? kvh : 0;
@@ -193,19 +208,9 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     const int n_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
     for (int s = early; s < STAGES - 1; ++s) issue_tile(s, n_rows);
 
-    // ---- Q^T as B operand: head = lane / 4, dims 2*(lane%4)+{0,1} (+8) of every 16-dim step ----
-    const int hq = lane >> 2;                 // head column this thread feeds
-    const int qd = (lane & 3) * 2;
-    unsigned qb[C::KSTEPS][2];
-    {
-        const T* qrow = reinterpret_cast<const T*>(a.q) + ((int64_t)b * a.H_q + kvh * G + (hq < G ? hq : 0)) * D;
+    if (hq >= G) {
 #pragma unroll
-        for (int kk = 0; kk < C::KSTEPS; ++kk) {
-            const unsigned lo = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd);
-            const unsigned hi = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd + 8);
-            qb[kk][0] = hq < G ? lo : 0u;
-            qb[kk][1] = hq < G ? hi : 0u;
-        }
+        for (int kk = 0; kk < C::KSTEPS; ++kk) { qb[kk][0] = 0u; qb[kk][1] = 0u; }
     }
     // accumulator-fragment coordinates: keys (or dims) lane/4 and lane/4 + 8, heads hc and hc + 1
     const int hc = (lane & 3) * 2;

@@ -48,8 +48,7 @@ struct AttnArgs {
 
 // Number of tokens request b attends over.  In a fused decode step that is one more than the
 // cache holds, unless the request is full (the token is then dropped, as by the append call).
-__device__ __forceinline__ int step_seq_len(const AttnArgs& a, int b, bool& has_new) {
-    const int S = a.seq_len[b];
+__device__ __forceinline__ int step_seq_len(const AttnArgs& a, int S /* = seq_len[b] */, bool& has_new) {
     has_new = a.step_append != 0 && S >= 0 && S < a.max_seq_len;
     return has_new ? S + 1 : S;
 }
