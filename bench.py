@@ -585,15 +585,20 @@ def oracle_baseline(synth, inputs, w, mode, sample=16, min_seconds=10.0):
         kw.update(mode=ora.MODE_DENSE)
     else:
         kw.update(mode=ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride_grid=w.stride)
-    reps, t0 = 0, time.perf_counter()
-    while True:
-        ora.decode(sub["q"], sub["k_cache"], sub["v_cache"], sub["seq_len"], sub["prompt_len"], **kw)
-        reps += 1
-        el = time.perf_counter() - t0
-        if el >= min_seconds or reps >= 1000:
-            break
+    def timed(seconds, **extra):
+        reps, t0 = 0, time.perf_counter()
+        while True:
+            ora.decode(sub["q"], sub["k_cache"], sub["v_cache"], sub["seq_len"], sub["prompt_len"], **kw, **extra)
+            reps += 1
+            el = time.perf_counter() - t0
+            if el >= seconds or reps >= 1000:
+                return reps, el
+
+    reps, el = timed(min_seconds)                         # all host threads (OpenMP over request x head)
+    reps1, el1 = timed(min_seconds / 4, n_threads=1)      # and one thread, for the per-core rate
     return {"value": round(n * reps / el, 2), "unit": UNIT, "cores": ora.num_threads(), "kind": "oracle",
-            "sample": "first %d requests of the batch, %d repetitions, %.1f s" % (n, reps, el)}
+            "sample": "first %d requests of the batch, %d repetitions, %.1f s" % (n, reps, el),
+            "single_thread_value": round(n * reps1 / el1, 2)}
 
 
 def run_reference(args):

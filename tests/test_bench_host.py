@@ -30,3 +30,12 @@ def test_workload_names_are_distinct():
     assert len(names) == 10
     w = synth.workload(5, batch=256)
     assert bench.workload_name(w, "sparse") in bench.NCU_TRAFFIC_BYTES
+
+
+def test_oracle_baseline_reports_all_threads_and_one_thread():
+    import torch
+    w = synth.workload(5, batch=2)
+    inputs = synth.make_inputs_device(w, torch.device("cpu"), seed=3)
+    res = bench.oracle_baseline(synth, inputs, w, "sparse", sample=2, min_seconds=0.5)
+    assert res["kind"] == "oracle" and res["cores"] >= 1 and res["unit"] == bench.UNIT
+    assert res["value"] > 0 and res["single_thread_value"] > 0
