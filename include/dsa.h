@@ -170,7 +170,7 @@ typedef struct dsa_diag_params {
 
 /* What a call will launch (filled by dsa_query_plan; for reporting and for tests). */
 typedef struct dsa_plan_info {
-    int32_t split_tokens;   /* kept tokens per thread block                                        */
+    int32_t split_tokens;   /* kept tokens per work item                                           */
     int32_t n_split;        /* splits per (request, kv head); 1 = results written directly         */
     int32_t launches;       /* kernels launched by the call (1, or 2 with the combine)             */
     int32_t grid_blocks;    /* thread blocks of the attention kernel                               */
@@ -180,6 +180,8 @@ typedef struct dsa_plan_info {
     int32_t tensor_cores;   /* 1: tensor-core kernel (bf16), one warp per work item;               */
                             /* 0: CUDA-core kernel (fp32), one 128-thread block per work item      */
     int32_t work_items;     /* (request, kv head, split) items                                     */
+    int32_t item_warps;     /* warps that share one work item (4 in small tensor-core launches,    */
+                            /* merged in shared memory; else 1)                                    */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);

@@ -54,7 +54,8 @@ class dsa_plan_info(ctypes.Structure):
     _fields_ = [("split_tokens", ctypes.c_int32), ("n_split", ctypes.c_int32),
                 ("launches", ctypes.c_int32), ("grid_blocks", ctypes.c_int32),
                 ("smem_bytes", ctypes.c_int32), ("tile_tokens", ctypes.c_int32),
-                ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32)]
+                ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32),
+                ("item_warps", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:

@@ -25,6 +25,7 @@ constexpr int kMaxDevices = 64;
 #ifndef DSA_TUNE_MMA_STAGES
 #define DSA_TUNE_MMA_STAGES 3
 #endif
+constexpr int kMmaItemWarps = 4;                   // warps per work item in small launches
 constexpr int kMmaStages = DSA_TUNE_MMA_STAGES;    // 16-key tiles in flight per warp (+1 being consumed)
 
 int env_int(const char* name, int fallback) {
@@ -64,6 +65,7 @@ struct Plan {
     int bitmap_words;
     bool mma;            // bf16: one warp per work item, tensor-core tiles
     int mma_warps;       // warps (= kv heads) per block that share one row list
+    int mma_kw;          // warps that share one work item (small launches), 1 or kMmaItemWarps
     int64_t grid;
     size_t smem;
     size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
@@ -94,15 +96,16 @@ struct KernelPick {
     // depend on the head (never with per-head masks or selection).
     template <int W>
     static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, kMmaStages, HM, SEL, W>::smem_bytes(chunk, bw); }
-    static size_t smem_mma(int w, int chunk, int bw) {
+    static size_t smem_mma(int w, int kw, int chunk, int bw) {
+        if (kw > 1) return smem_mma_w<kMmaItemWarps>(chunk, bw);      // one ring per warp either way
         if constexpr (!HM && !SEL) {
             if (w == 2) return smem_mma_w<2>(chunk, bw);
         }
         return smem_mma_w<1>(chunk, bw);
     }
-    template <int W, bool APPEND>
+    template <int W, bool APPEND, int KW>
     static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND>;
+        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>;
         static bool configured[kMaxDevices] = {};
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -112,24 +115,26 @@ struct KernelPick {
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
         }
-        return launch_pdl(kern, (unsigned)grid, 32 * W, smem_bytes, st, a);
+        return launch_pdl(kern, (unsigned)grid, 32 * W * KW, smem_bytes, st, a);
     }
     // `append`: the fused decode step (the kernel reads the current token from a.k_new / a.v_new)
     template <bool APPEND>
-    static cudaError_t launch_mma_a(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
+    static cudaError_t launch_mma_a(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
+                                    cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
+            if (kw > 1) return launch_mma_w<1, APPEND, kMmaItemWarps>(a, items, smem_bytes, st);
             if constexpr (!HM && !SEL) {
-                if (w == 2) return launch_mma_w<2, APPEND>(a, items / 2, smem_bytes, st);
+                if (w == 2) return launch_mma_w<2, APPEND, 1>(a, items / 2, smem_bytes, st);
             }
-            return launch_mma_w<1, APPEND>(a, items, smem_bytes, st);
+            return launch_mma_w<1, APPEND, 1>(a, items, smem_bytes, st);
         } else {
             return cudaErrorInvalidValue;
         }
     }
-    static cudaError_t launch_mma(int w, const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st,
-                                  bool append) {
-        return append ? launch_mma_a<true>(w, a, items, smem_bytes, st)
-                      : launch_mma_a<false>(w, a, items, smem_bytes, st);
+    static cudaError_t launch_mma(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
+                                  cudaStream_t st, bool append) {
+        return append ? launch_mma_a<true>(w, kw, a, items, smem_bytes, st)
+                      : launch_mma_a<false>(w, kw, a, items, smem_bytes, st);
     }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
         auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
@@ -267,6 +272,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     // DSA_CUDA_CORES=1 forces the latter for bf16 too (comparison runs).
     pl->mma = p->dtype == DSA_BF16 && env_int("DSA_CUDA_CORES", 0) == 0;
     pl->mma_warps = 1;
+    pl->mma_kw = 1;
     if (pl->mma) {
         pl->tile = MMA_KEYS;
         pl->stages = kMmaStages;
@@ -286,14 +292,27 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         const int64_t target = (pl->mma ? 6 : 4) * kNumSMs;        // a work item is a warp / a 4-warp block
         int64_t want_split = std::max<int64_t>(1, (target + pairs - 1) / pairs);
         want_split = std::min<int64_t>(want_split, std::max<int64_t>(1, bound / (pl->mma ? 96 : 128)));
-        want_split = std::max<int64_t>(want_split, (bound + MAX_CHUNK - 1) / MAX_CHUNK);
+        int max_chunk = MAX_CHUNK;
+        if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK && env_int("DSA_ITEM_WARPS", 1) != 0) {
+            // Too few pairs to fill the device, and a request fits one (long) row list: the
+            // tensor-core kernel puts kMmaItemWarps warps on one work item and merges them in
+            // shared memory -- the same parallelism without partial results and, up to
+            // kMmaItemWarps pieces, without the combine launch.  Those blocks hold four rings, so
+            // a list of twice the usual length costs no occupancy.  (Longer requests need the
+            // combine anyway; there the merge on top of it measured as a small loss.)
+            pl->mma_kw = kMmaItemWarps;
+            pl->mma_warps = 1;
+            want_split = (want_split + kMmaItemWarps - 1) / kMmaItemWarps;
+            max_chunk = 2 * MAX_CHUNK;
+        }
+        want_split = std::max<int64_t>(want_split, (bound + max_chunk - 1) / max_chunk);
         // Requests too long for one row list are split anyway; when the (request, kv head) pairs
         // alone fill half the device's warp slots, ~512-row items balance better across the SMs
         // than ~900-row ones (measured on dense calls: +3-10 % at 640-4096 pairs, a loss below).
-        if (bound > MAX_CHUNK && pairs >= 4 * kNumSMs)
+        if (pl->mma_kw == 1 && bound > MAX_CHUNK && pairs >= 4 * kNumSMs)
             want_split = std::max<int64_t>(want_split, (bound + 511) / 512);
         const int64_t c = (bound + want_split - 1) / want_split;
-        chunk = std::min(MAX_CHUNK, round_up((int)c, pl->tile));
+        chunk = std::min(max_chunk, round_up((int)c, pl->tile));
     }
     pl->chunk = chunk;
     pl->n_split = (int)((bound + chunk - 1) / chunk);
@@ -302,7 +321,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
 
     dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
-        smem_probe = pl->mma ? P::smem_mma(pl->mma_warps, pl->chunk, pl->bitmap_words)
+        smem_probe = pl->mma ? P::smem_mma(pl->mma_warps, pl->mma_kw, pl->chunk, pl->bitmap_words)
                              : P::smem(pl->chunk, pl->bitmap_words);
         return DSA_OK;
     });
@@ -439,7 +458,7 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     cudaError_t err = cudaSuccess;
     rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, pl.select, [&](auto pick) -> int32_t {
         using P = decltype(pick);
-        err = pl.mma ? P::launch_mma(pl.mma_warps, a, pl.grid, pl.smem, st, step && pl.mma)
+        err = pl.mma ? P::launch_mma(pl.mma_warps, pl.mma_kw, a, pl.grid, pl.smem, st, step && pl.mma)
                      : P::launch(a, pl.grid, pl.smem, st);
         return DSA_OK;
     });
@@ -514,6 +533,7 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->tile_tokens = pl.tile;
     info->tensor_cores = pl.mma ? 1 : 0;
     info->work_items = (int32_t)pl.grid;
+    info->item_warps = pl.mma ? pl.mma_kw : 1;
     info->stages = pl.stages;
     return DSA_OK;
 }

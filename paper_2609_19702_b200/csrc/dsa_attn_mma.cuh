@@ -87,13 +87,20 @@ struct MmaItemCfg {
 // read from k_new / v_new wherever the row list names its position, and the warps of split 0
 // write them to the cache (nobody reads that slot in this launch: with a bounded cache it belonged
 // to a token that has left the window).
-template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false>
-__global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) {
-    using C = MmaCfg<D, G, STAGES, HEADMASK, SELECT, W>;
+//
+// KW > 1: small launches.  When the (request, kv head) pairs are too few to fill the device, KW
+// warps share one work item instead of the item being cut into KW splits with a combine launch
+// behind them: they build the row list together, warp k streams tiles k, k + KW, ... through its
+// own ring, and the partial softmax states are merged through shared memory at the end.
+template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false, int KW = 1>
+__global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArgs a) {
+    using C = MmaCfg<D, G, STAGES, HEADMASK, SELECT, W * KW>;   // one ring per warp
     using IC = MmaItemCfg<D, G, HEADMASK, SELECT>;
     using T = __nv_bfloat16;
     constexpr unsigned FULL = 0xffffffffu;
+    constexpr int NW = W * KW;                            // warps per block
     static_assert(W == 1 || (!HEADMASK && !SELECT), "a shared row list needs a head-independent mask");
+    static_assert(W == 1 || KW == 1, "several warps per head only with one head per block");
 
     // Programmatic launch on both sides: a combine kernel queued behind this grid may be scheduled
     // from now on (it waits for this grid to finish before it reads anything), and this grid may
@@ -102,16 +109,18 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ int s_warp[W];
+    __shared__ int s_warp[NW];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int hw = KW == 1 ? warp : 0;                    // this warp's head within the block
+    const int wk = KW == 1 ? 0 : warp;                    // its rank among the warps of that head
     unsigned char* ring = smem + warp * (STAGES * C::SLOT_BYTES);
-    const RowList list = RowList::carve<IC>(smem + W * STAGES * C::SLOT_BYTES, a.chunk);
-    unsigned* bitmaps = reinterpret_cast<unsigned*>(smem + W * STAGES * C::SLOT_BYTES + C::list_bytes(a.chunk));
+    const RowList list = RowList::carve<IC>(smem + NW * STAGES * C::SLOT_BYTES, a.chunk);
+    unsigned* bitmaps = reinterpret_cast<unsigned*>(smem + NW * STAGES * C::SLOT_BYTES + C::list_bytes(a.chunk));
 
     // kv heads vary fastest across the grid: the warps that run together read the same tokens
     // of neighbouring heads, i.e. neighbouring memory.
     const int hblocks = a.H_kv / W;
-    const int kvh = (blockIdx.x % hblocks) * W + warp;
+    const int kvh = (blockIdx.x % hblocks) * W + hw;
     const int split = (blockIdx.x / hblocks) % a.n_split;
     const int b = blockIdx.x / (hblocks * a.n_split);
 
@@ -133,7 +142,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     bool has_new = false;
     const int S_step = APPEND ? step_seq_len(a, seq_raw, has_new) : seq_raw;
     const ReqMask m = req_mask_setup(a.mask, S_step, prompt_raw, a.max_seq_len);
-    auto sync_builders = [&]() { if (W == 1) __syncwarp(); else __syncthreads(); };
+    auto sync_builders = [&]() { if (NW == 1) __syncwarp(); else __syncthreads(); };
     // W > 1: one list for all the block's heads, built without a head offset (kv head "0")
     const int list_kvh = W == 1 ? kvh : 0;
     const int64_t head_bytes = W == 1 ? 0 : (int64_t)kvh * a.stride_head * 2;
@@ -145,7 +154,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     int64_t off_new = 0;
     int new_r = -1;                                       // its row in this item's list, once known
     uint4 new_chunk = make_uint4(0u, 0u, 0u, 0u);
-    const bool store_new = APPEND && has_new && split == 0 && lane < 2 * C::CPR;
+    const bool store_new = APPEND && has_new && split == 0 && wk == 0 && lane < 2 * C::CPR;
     if (APPEND && has_new) {
         const int64_t row_bytes = ((int64_t)b * a.H_kv + kvh) * C::ROW_BYTES;
         knew_row = reinterpret_cast<const unsigned char*>(a.k_new) + row_bytes;
@@ -159,15 +168,17 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
 
     // ---- staging: this warp's own ring of 16-key tiles ---------------------------------------
     // rows_ready: rows of the list that exist so far (tiles below it can be issued)
+    // `tile` counts this warp's own tiles; it is tile wk + tile * KW of the item
     auto issue_tile = [&](int tile, int rows_ready) {
-        if (tile * MMA_KEYS < rows_ready) {
+        const int row0 = (wk + tile * KW) * MMA_KEYS;
+        if (row0 < rows_ready) {
             unsigned char* ks = ring + (tile % STAGES) * C::SLOT_BYTES;
             unsigned char* vs = ks + C::TILE_BYTES;
 #pragma unroll
             for (int i = 0; i < MMA_KEYS * C::CPR / 32; ++i) {
                 const int idx = i * 32 + lane;
                 const int row = idx / C::CPR, c = idx % C::CPR;
-                const int r = tile * MMA_KEYS + row;
+                const int r = row0 + row;
                 const bool valid = r < rows_ready;
                 const int64_t off = valid ? list.rowoff[r] * 2 + head_bytes + c * 16 : 0;
                 const int dst = row * C::ROW_BYTES + ((c ^ (row & 7)) * 16);       // swizzled chunk
@@ -186,26 +197,31 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     // Phase A of the row list: the rows that need no scan (prompt, old sinks, unmasked window).
     // The first tiles of the ring are issued from them right away, so that the memory stream is
     // already running while phase B (mask bitmaps, window scan, block-table lookups) is computed.
-    const int n_direct = W == 1 ? build_rows_direct<IC, 32>(a, m, b, list_kvh, split, list)
-                                : build_rows_direct<IC, 32 * W>(a, m, b, list_kvh, split, list);
+    const int n_direct = build_rows_direct<IC, 32 * NW>(a, m, b, list_kvh, split, list);
     sync_builders();
     // whole tiles inside phase A (fused step: never the newest row, which may not be in the cache)
-    const int early = min(STAGES - 1, (n_direct - (APPEND ? 1 : 0)) / MMA_KEYS);
+    // that are this warp's
+    const int whole_a = (n_direct - (APPEND ? 1 : 0)) / MMA_KEYS;
+    const int early = min(STAGES - 1, whole_a > wk ? (whole_a - wk + KW - 1) / KW : 0);
     for (int s = 0; s < early; ++s) issue_tile(s, n_direct);
-    const int n_rows = W == 1
+    const int n_rows = NW == 1
         ? build_rows_scanned<IC, WarpSync, 32>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct)
-        : build_rows_scanned<IC, BlockSync, 32 * W>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct);
+        : build_rows_scanned<IC, BlockSync, 32 * NW>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct);
     if (store_new) {
         unsigned char* base = const_cast<unsigned char*>(lane < C::CPR ? kbase : vbase);
         const int c = lane < C::CPR ? lane : lane - C::CPR;
         *reinterpret_cast<uint4*>(base + (off_new + (int64_t)kvh * a.stride_head) * 2 + c * 16) = new_chunk;
     }
-    if (n_rows <= 0) { write_empty_item<IC, 32>(a, m, b, kvh, split, lane); return; }
+    if (n_rows <= 0) {
+        if (wk == 0) write_empty_item<IC, 32>(a, m, b, kvh, split, lane);
+        return;
+    }
     sync_builders();                                   // the last barrier: from here on warps run free
     // kept positions ascend, so the token being decoded can only be this item's last row
     if (APPEND && has_new && list.rowoff[n_rows - 1] == off_new + (int64_t)list_kvh * a.stride_head)
         new_r = n_rows - 1;
-    const int n_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
+    const int item_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
+    const int n_tiles = item_tiles > wk ? (item_tiles - wk + KW - 1) / KW : 0;      // this warp's
     for (int s = early; s < STAGES - 1; ++s) issue_tile(s, n_rows);
 
     if (hq >= G) {
@@ -246,7 +262,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
             mma_bf16_16816(s, af, qb[kk][0], qb[kk][1]);
         }
         // s[0]: (key kr, head hc)  s[1]: (kr, hc+1)  s[2]: (kr+8, hc)  s[3]: (kr+8, hc+1)
-        const int r0 = tile * MMA_KEYS + kr, r1 = r0 + 8;
+        const int r0 = (wk + tile * KW) * MMA_KEYS + kr, r1 = r0 + 8;
         const bool v0 = r0 < n_rows, v1 = r1 < n_rows;
         unsigned bits0 = 0xffu, bits1 = 0xffu;
         if (HEADMASK) { bits0 = v0 ? list.hbits[r0] : 0u; bits1 = v1 ? list.hbits[r1] : 0u; }
@@ -294,23 +310,77 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
     }
     cp_async_wait<0>();
 
-    // ---- finish: sums over the key lanes, normalise, write ------------------------------------
+    // ---- finish: sums over the key lanes, merge the warps of the item, normalise, write --------
+    float ltot[2], bv[2];
+    int bp[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
         float l = lpart[j];
         l += __shfl_xor_sync(FULL, l, 4);
         l += __shfl_xor_sync(FULL, l, 8);
         l += __shfl_xor_sync(FULL, l, 16);
-        float bv = bestv[j];
-        int bp = bestp[j];
+        ltot[j] = l;
+        bv[j] = bestv[j];
+        bp[j] = bestp[j];
         if (SELECT) {
 #pragma unroll
             for (int off = 4; off <= 16; off <<= 1) {
-                const float ov = __shfl_xor_sync(FULL, bv, off);
-                const int op = __shfl_xor_sync(FULL, bp, off);
-                if (ov < bv || (ov == bv && op < bp)) { bv = ov; bp = op; }
+                const float ov = __shfl_xor_sync(FULL, bv[j], off);
+                const int op = __shfl_xor_sync(FULL, bp[j], off);
+                if (ov < bv[j] || (ov == bv[j] && op < bp[j])) { bv[j] = ov; bp[j] = op; }
             }
         }
+    }
+    if (KW > 1) {
+        // Every warp holds its state in the same fragment layout, so the merge is element-wise:
+        // warps 1.. leave theirs in shared memory (the rings are free now), warp 0 folds them in.
+        constexpr int REC = C::MTILES * 4 + 8;            // floats per lane: o, m[2], l[2], best value[2], best position[2]
+        float* rec = reinterpret_cast<float*>(smem);
+        __syncthreads();                                  // all rings drained and consumed
+        if (wk > 0) {
+            float* mine = rec + (size_t)(wk - 1) * REC * 32 + lane;
+#pragma unroll
+            for (int mt = 0; mt < C::MTILES; ++mt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) mine[(mt * 4 + e) * 32] = o[mt][e];
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                mine[(C::MTILES * 4 + j) * 32] = mrun[j];
+                mine[(C::MTILES * 4 + 2 + j) * 32] = ltot[j];
+                mine[(C::MTILES * 4 + 4 + j) * 32] = bv[j];
+                mine[(C::MTILES * 4 + 6 + j) * 32] = __int_as_float(bp[j]);
+            }
+        }
+        __syncthreads();
+        if (wk > 0) return;
+        for (int w = 1; w < KW; ++w) {
+            const float* other = rec + (size_t)(w - 1) * REC * 32 + lane;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const float m_o = other[(C::MTILES * 4 + j) * 32];
+                const float l_o = other[(C::MTILES * 4 + 2 + j) * 32];
+                const float mnew = fmaxf(mrun[j], m_o);
+                const float msafe = mnew == -INFINITY ? 0.f : mnew;
+                const float c0 = fast_exp2(mrun[j] - msafe), c1 = fast_exp2(m_o - msafe);
+                ltot[j] = ltot[j] * c0 + l_o * c1;
+                mrun[j] = mnew;
+#pragma unroll
+                for (int mt = 0; mt < C::MTILES; ++mt) {
+                    o[mt][j] = o[mt][j] * c0 + other[(mt * 4 + j) * 32] * c1;
+                    o[mt][2 + j] = o[mt][2 + j] * c0 + other[(mt * 4 + 2 + j) * 32] * c1;
+                }
+                if (SELECT) {
+                    const float ov = other[(C::MTILES * 4 + 4 + j) * 32];
+                    const int op = __float_as_int(other[(C::MTILES * 4 + 6 + j) * 32]);
+                    if (ov < bv[j] || (ov == bv[j] && op < bp[j])) { bv[j] = ov; bp[j] = op; }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const float l = ltot[j];
         const int h = hc + j;
         if (h < G) {
             const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -333,9 +403,9 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_mma_kernel(const AttnArgs a) 
                 if (a.n_split > 1) a.lse_part[row * a.n_split + split] = lse;
                 else a.lse[row] = lse;
                 if (SELECT) {
-                    const int off = bp == 0x7fffffff ? -1 : (m.S - 1) - bp;
+                    const int off = bp[j] == 0x7fffffff ? -1 : (m.S - 1) - bp[j];
                     if (a.n_split > 1) {
-                        a.sel_val_part[row * a.n_split + split] = bv;
+                        a.sel_val_part[row * a.n_split + split] = bv[j];
                         a.sel_off_part[row * a.n_split + split] = off;
                         a.sel_k[row] = m.sel_k;
                     } else if (m.sel_k >= 0) {

@@ -9,7 +9,7 @@
 namespace dsa {
 
 constexpr int NT = 128;          // compute threads per block (4 warps)
-constexpr int MAX_CHUNK = 1024;  // kept rows one work item can hold in its row list
+constexpr int MAX_CHUNK = 1024;  // kept rows one work item can hold in its row list (twice that when four warps share it)
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -28,7 +28,7 @@ struct AttnArgs {
     int B, H_q, H_kv;
     float scale_log2;            // sm_scale * log2(e)
     MaskArgs mask;
-    int chunk;                   // kept rows per split (multiple of the tile, <= MAX_CHUNK)
+    int chunk;                   // kept rows per split (multiple of the tile; see MAX_CHUNK)
     int n_split;
     int n_items;                 // B * H_kv * n_split work items
     void* out;                   // n_split == 1: [B, H_q, D] in T

@@ -29,12 +29,17 @@ def _pinned_step(prob):
     return h
 
 
-@pytest.mark.parametrize("index,batch,mode", [(2, None, "sparse"), (2, None, "dense"), (5, 3, "sparse"),
-                                              (5, 3, "dense"), (4, None, "sparse")])
-def test_host_mapped_step_matches_oracle_and_device_call(dsa, index, batch, mode):
+# (config, batch, mode, forced rows per split): plans with one work item per (request, kv head) read q
+# from the host buffer; plans with several splits stage it on the device first
+CASES = [(2, None, "sparse", 0), (2, None, "dense", 0), (5, 3, "sparse", 0), (5, 3, "dense", 0),
+         (4, None, "sparse", 0), (5, 3, "sparse", 96), (2, None, "dense", 128)]
+
+
+@pytest.mark.parametrize("index,batch,mode,split", CASES)
+def test_host_mapped_step_matches_oracle_and_device_call(dsa, index, batch, mode, split):
     w = synth.workload(index) if batch is None else synth.workload(index, batch=batch)
     inp = synth.make_inputs(w)
-    prob = dsa.problem_from_host(inp)
+    prob = dsa.problem_from_host(inp, split_tokens=split)
     diag = None if mode == "dense" else dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
     ref_out, ref_lse = dsa.alloc_outputs(prob)
     ws = dsa.alloc_workspace(prob, diag)
@@ -71,11 +76,11 @@ def test_host_mapped_step_matches_oracle_and_device_call(dsa, index, batch, mode
 def test_host_mapped_plans_cover_both_q_paths(dsa):
     """The cases above must exercise the direct read of q (one split) and the staged copy (several)."""
     seen = set()
-    for index, batch, sparse in ((2, None, True), (2, None, False), (5, 3, True), (4, None, True)):
+    for index, batch, mode, split in CASES:
         w = synth.workload(index) if batch is None else synth.workload(index, batch=batch)
         inp = synth.make_inputs(w)
-        prob = dsa.problem_from_host(inp)
-        diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra) if sparse else None
+        prob = dsa.problem_from_host(inp, split_tokens=split)
+        diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra) if mode == "sparse" else None
         seen.add(min(dsa.dsa_query_plan(prob, diag).n_split, 2))
     assert seen == {1, 2}
 

@@ -1,0 +1,96 @@
+"""Small launches of the tensor-core kernel put four warps on one work item and merge their
+softmax states in shared memory instead of splitting the item and combining in a second launch.
+
+Checked here: the plan really takes that path for the small configurations, every mask mode on it
+matches the oracle (kept sets are untouched by it), requests so short that some of the four warps
+get no tile at all are handled, and the result -- the entries picked by the fused selection
+included, which the selection tests pin to the oracle on the one-warp plan -- agrees with the
+one-warp-per-item plan of the same library within the summation-order difference."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as ora
+from paper_2609_19702_b200 import synth
+from tests import util
+from tests.test_gpu_parity import _check_all_modes
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dsa():
+    from paper_2609_19702_b200 import binding
+    return binding
+
+
+def _plan(dsa, inp, diag):
+    return dsa.dsa_query_plan(dsa.problem_from_host(inp), diag)
+
+
+@pytest.mark.parametrize("name,make", [
+    ("config3, batch 2", lambda: synth.workload(3, batch=2)),
+    ("config4 GQA, batch 3", lambda: synth.workload(4, batch=3)),
+    ("config5 paged, batch 2", lambda: synth.workload(5, batch=2)),
+    ("head_dim 64, 3 kv heads x 2", lambda: synth.Workload("kw", 91, 4, 6, 3, 64, 150, 20, 19, 1, 200, 60, 1, 400)),
+])
+def test_all_masks_on_the_shared_item_path(dsa, name, make):
+    w = make()
+    inp = synth.make_inputs(w)
+    grid = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    # (longer bounds still split, each split then shared by four warps: covered by the same cases)
+    for diag in (grid, dsa.Diag(dsa.DSA_MASK_WINDOW, w.window)):
+        plan = _plan(dsa, inp, diag)
+        assert plan.tensor_cores == 1 and plan.item_warps == 4, name
+        assert plan.launches == (1 if plan.n_split == 1 else 2)
+    heads = (1, w.num_q_heads) if w.num_q_heads != w.num_kv_heads else (w.num_q_heads,)
+    _check_all_modes(dsa, inp, list_heads=heads, seed=7, what=name)
+
+
+def test_requests_shorter_than_one_tile_per_warp(dsa):
+    # bound 40 + 300 rows, but most requests hold 1..40 rows: warps 1-3 of their items stay idle
+    w = synth.Workload("short", 92, 12, 8, 8, 128, 0, 20, 15, 0, 300, 80, 1, 300)
+    inp = synth.make_inputs(w, poison=False)              # (lengths are rewritten below: no NaN tail)
+    inp["position"][:8] = np.arange(1, 9) * 5
+    inp["seq_len"][:8] = inp["prompt_len"][:8] + inp["position"][:8]
+    diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    assert _plan(dsa, inp, diag).item_warps == 4
+    _check_all_modes(dsa, inp, list_heads=(8,), seed=3, what="short requests")
+
+
+def test_shared_item_path_agrees_with_one_warp_per_item(dsa):
+    w = synth.workload(5, batch=4)
+    inp = synth.make_inputs(w)
+    prob = dsa.problem_from_host(inp)
+    rng = np.random.default_rng(4)
+    trace = synth.random_valid_trace(rng, w.window, w.n_att, (w.batch, w.num_q_heads))
+    results = {}
+    for setting in ("1", "0"):
+        os.environ["DSA_ITEM_WARPS"] = setting
+        try:
+            outs = []
+            for diag in (None, dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra),
+                         dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att,
+                                  skip_offsets=torch.from_numpy(trace.copy()).cuda(), select=True)):
+                plan = dsa.dsa_query_plan(prob, diag)
+                if diag is not None:
+                    assert plan.item_warps == (4 if setting == "1" else 1)
+                out, lse = dsa.alloc_outputs(prob)
+                ws = dsa.alloc_workspace(prob, diag)
+                if diag is None:
+                    dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+                else:
+                    dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+                torch.cuda.synchronize()
+                outs.append((out.float().cpu(), lse.cpu(), None if diag is None else diag.skip_offsets))
+            results[setting] = outs
+        finally:
+            os.environ.pop("DSA_ITEM_WARPS", None)
+    for (o1, l1, t1), (o0, l0, t0) in zip(results["1"], results["0"]):
+        assert torch.allclose(o1, o0, atol=2e-2, rtol=2e-2)
+        assert torch.allclose(l1, l0, atol=1e-4, rtol=0)
+        if t1 is not None:
+            # the selected distances (one new trace entry per head) must be the same keys
+            assert torch.equal(t1.cpu(), t0.cpu())
