@@ -116,3 +116,53 @@ def test_plan_sizes(dsa):
     # a few requests with long sequences are split to fill the machine
     rc, info = _plan(dsa, _problem(dsa, batch=1))
     assert rc == 0 and info.grid_blocks >= 148
+
+
+def test_small_launch_plan_shares_items_between_warps(dsa):
+    # 8 requests x 8 kv heads cannot fill the device: four warps per item, no split, one launch
+    rc, info = _plan(dsa, _problem(dsa, batch=8), _diag(dsa))
+    assert rc == 0 and info.tensor_cores == 1 and info.item_warps == 4
+    assert info.n_split == 1 and info.launches == 1 and info.split_tokens >= 64 + 410
+    # the same requests without a mask are longer than one row list: split, one warp per item
+    rc, info = _plan(dsa, _problem(dsa, batch=8))
+    assert rc == 0 and info.item_warps == 1 and info.n_split > 1 and info.launches == 2
+    # a full device keeps one warp per item
+    rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,
+                                   max_prompt_len=200), _diag(dsa, window=512, n_att=208, grid_w=64))
+    assert rc == 0 and info.item_warps == 1
+    # the CUDA-core kernel (float32) has no such form
+    rc, info = _plan(dsa, _problem(dsa, batch=8, dtype=dsa.DSA_F32), _diag(dsa))
+    assert rc == 0 and info.tensor_cores == 0 and info.item_warps == 1
+
+
+def test_newer_entry_points_validate_before_touching_a_device(dsa):
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    p, d = _problem(dsa), _diag(dsa)
+    fake = ctypes.c_void_p(0x50000)
+    # fused step: the current token's rows are required, and must be 16-byte aligned
+    step = lib.dsa_decode_step
+    step.argtypes = [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p]
+    assert step(ctypes.byref(p), ctypes.byref(d), None, fake, fake, fake, None, 0, None) == -1
+    assert step(ctypes.byref(p), ctypes.byref(d), fake, None, fake, fake, None, 0, None) == -1
+    assert step(ctypes.byref(p), ctypes.byref(d), ctypes.c_void_p(0x50004), fake, fake, fake, None, 0, None) == -1
+    bad = _problem(dsa, head_dim=96)
+    assert step(ctypes.byref(bad), ctypes.byref(d), fake, fake, fake, fake, None, 0, None) == -2
+    # seq_len advance
+    adv = lib.dsa_advance_seq_len
+    adv.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
+    assert adv(None, 4, 100, None) == -1
+    assert adv(fake, -1, 100, None) == -1
+    assert adv(fake, 4, -5, None) == -1
+    assert adv(None, 0, 100, None) == 0
+    # host-buffer steps: every host pointer is required; pointers that are not page-locked host
+    # memory the device can address are refused (here: no such memory exists at all)
+    mapped = lib.dsa_decode_attention_host_mapped
+    mapped.argtypes = [ctypes.c_void_p] * 9 + [ctypes.c_size_t, ctypes.c_void_p]
+    host = (ctypes.c_char * 4096)()
+    hp = ctypes.cast(host, ctypes.c_void_p)
+    assert mapped(ctypes.byref(p), ctypes.byref(d), None, hp, hp, None, hp, hp, None, 0, None) == -1
+    assert mapped(ctypes.byref(p), ctypes.byref(d), hp, hp, hp, None, hp, hp, None, 0, None) == -1
+    assert mapped(ctypes.byref(p), ctypes.byref(d), hp, hp, hp, hp, hp, hp, None, 0, None) == -1   # table without a paged cache
+    host_io = lib.dsa_decode_attention_host_io
+    host_io.argtypes = [ctypes.c_void_p] * 11 + [ctypes.c_size_t, ctypes.c_void_p]
+    assert host_io(ctypes.byref(p), ctypes.byref(d), None, hp, hp, None, fake, fake, hp, hp, None, 0, None) == -1

@@ -60,8 +60,13 @@ def test_requests_shorter_than_one_tile_per_warp(dsa):
     _check_all_modes(dsa, inp, list_heads=(8,), seed=3, what="short requests")
 
 
-def test_shared_item_path_agrees_with_one_warp_per_item(dsa):
-    w = synth.workload(5, batch=4)
+@pytest.mark.parametrize("name,make,splits", [
+    ("paged, one split", lambda: synth.workload(5, batch=4), 1),
+    # 600 kept rows for 4 pairs: two splits, each shared by four warps, then the combine kernel
+    ("long list, two splits", lambda: synth.Workload("kw2", 94, 2, 4, 2, 128, 200, 30, 29, 1, 600, 400, 500, 880), 2),
+])
+def test_shared_item_path_agrees_with_one_warp_per_item(dsa, name, make, splits):
+    w = make()
     inp = synth.make_inputs(w)
     prob = dsa.problem_from_host(inp)
     rng = np.random.default_rng(4)
@@ -76,7 +81,9 @@ def test_shared_item_path_agrees_with_one_warp_per_item(dsa):
                                   skip_offsets=torch.from_numpy(trace.copy()).cuda(), select=True)):
                 plan = dsa.dsa_query_plan(prob, diag)
                 if diag is not None:
-                    assert plan.item_warps == (4 if setting == "1" else 1)
+                    assert plan.item_warps == (4 if setting == "1" else 1), name
+                    if setting == "1":
+                        assert plan.n_split == splits, name
                 out, lse = dsa.alloc_outputs(prob)
                 ws = dsa.alloc_workspace(prob, diag)
                 if diag is None:
