@@ -35,6 +35,7 @@ METRIC = "decode_attention_queries_per_sec"
 UNIT = "queries/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 << 20
 # DRAM bytes per launch of the timed kernel from an ncu capture (see profiles/), keyed by the
 # workload string of the JSON line; None until a capture of that exact launch exists.
 NCU_TRAFFIC_BYTES = {
@@ -191,6 +192,33 @@ def time_calls(torch, fn, steps, warmup, sampler=None, barrier=None):
         torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
     return e0.elapsed_time(e1) / 1e3, clocks          # seconds for `steps` calls
+
+
+def time_calls_flushed(torch, fn, steps, warmup, flush, sampler=None, barrier=None):
+    """Like time_calls for working sets that would stay in L2: a write larger than L2 precedes every
+    call and only the calls are timed (one event pair each, summed)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+        torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    pairs = []
+    for _ in range(steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    return sum(a.elapsed_time(b) for a, b in pairs) / 1e3, clocks
 
 
 def time_flushed(torch, fn, flush, iters=30, warmup=3):
@@ -440,18 +468,9 @@ def run_ours(args):
             return (lambda: dsa.dsa_decode_attention_dense(prob, out, lse, ws)), plan, diag
         return (lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)), plan, diag
 
-    # ---- the timed step ------------------------------------------------------------------
     call, plan, diag = make_call(args.mode, w)
-    sampler = ClockSampler(local_rank)
-    secs, clocks = time_calls(torch, call, args.steps, args.warmup, sampler, barrier)
-    t = torch.tensor([secs], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    secs_max = float(t.item())
-    ms_per_step = secs_max / args.steps * 1e3
-    value = world * w.batch * args.steps / secs_max
 
-    # ---- roofline of the attention kernel (rank-local numbers) ----------------------------
+    # ---- algorithmic bytes of one step (rank-local; also decides how L2 is kept out of the timing)
     idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, inputs["max_seq_len"])
     torch.cuda.synchronize()
     if inputs["block_table"] is not None:
@@ -462,6 +481,27 @@ def run_ours(args):
         blocks_touched = 0
     del idx
     abytes, kept_rows = algorithmic_bytes(w, host, args.mode, blocks_touched)
+
+    # ---- the timed step ------------------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    flush_l2 = abytes < 2 * L2_BYTES
+    if flush_l2:
+        flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+        secs, clocks = time_calls_flushed(torch, call, args.steps, args.warmup, flush, sampler, barrier)
+        del flush
+        l2_note = ("working set (%.3f GB per step) would stay in the %d MB L2: a %d MB write precedes every timed "
+                   "call and only the calls are timed" % (abytes / 1e9, L2_BYTES >> 20, 4 * L2_BYTES >> 20))
+    else:
+        secs, clocks = time_calls(torch, call, args.steps, args.warmup, sampler, barrier)
+        l2_note = "inputs larger than L2: each step reads %.2f GB of distinct K/V" % (abytes / 1e9)
+    t = torch.tensor([secs], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    secs_max = float(t.item())
+    ms_per_step = secs_max / args.steps * 1e3
+    value = world * w.batch * args.steps / secs_max
+
+    # ---- roofline of the attention kernel (rank-local numbers) ----------------------------
     peak, peak_kind = measured_peak()
     launch_secs = secs / args.steps                       # one attention launch (+ combine) per step
     achieved = abytes / launch_secs / 1e9
@@ -482,8 +522,13 @@ def run_ours(args):
             todo.append(("sparse", synth.workload(5, batch=w.batch, window=1024, n_att=416)))
         for mode, ww in todo:
             vcall, vplan, _ = make_call(mode, ww)
-            vsecs, _ = time_calls(torch, vcall, vsteps, 3)
             vb, _ = algorithmic_bytes(ww, host, mode, 0)
+            if vb < 2 * L2_BYTES:                           # same rule as the timed step
+                vflush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+                vsecs, _ = time_calls_flushed(torch, vcall, vsteps, 3, vflush)
+                del vflush
+            else:
+                vsecs, _ = time_calls(torch, vcall, vsteps, 3)
             key = "dense" if mode == "dense" else "sparse_w%d_a%d" % (ww.window, ww.n_att)
             variants[key] = {"ms_per_step": round(vsecs / vsteps * 1e3, 4),
                              "queries_per_sec": round(w.batch * vsteps / vsecs, 1),
@@ -557,7 +602,7 @@ def run_ours(args):
             "data": "synthetic",
             "config": {"workload": name, "global_batch": world * w.batch,
                        "kept_rows_per_kv_head_mean": round(kept_rows / w.batch, 1),
-                       "l2": "inputs larger than L2: each step reads %.2f GB of distinct K/V" % (abytes / 1e9),
+                       "l2": l2_note,
                        "parallelism": "requests sharded over %d GPU(s), no collective" % world,
                        "plan": {"split_tokens": plan.split_tokens, "n_split": plan.n_split,
                                 "grid_blocks": plan.grid_blocks, "smem_bytes": plan.smem_bytes,
