@@ -291,19 +291,28 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         const int64_t pairs = (int64_t)std::max(p->batch, 1) * p->num_kv_heads;
         const int64_t target = (pl->mma ? 6 : 4) * kNumSMs;        // a work item is a warp / a 4-warp block
         int64_t want_split = std::max<int64_t>(1, (target + pairs - 1) / pairs);
+        // From half the warp slots on, one whole item per warp in a single wave beats two splits
+        // that spill into a second wave (640-864 pairs of ~400 rows: 30-35 us against 36-43 us).
+        if (pl->mma && pairs >= 4 * kNumSMs) want_split = 1;
         want_split = std::min<int64_t>(want_split, std::max<int64_t>(1, bound / (pl->mma ? 96 : 128)));
         int max_chunk = MAX_CHUNK;
+        // Too few pairs to fill the device, and a request fits one (long) row list: the
+        // tensor-core kernel puts kMmaItemWarps warps on one work item and merges them in shared
+        // memory -- the same parallelism without partial results and, up to kMmaItemWarps pieces,
+        // without the combine launch.  Those blocks hold four rings, so a list of twice the usual
+        // length costs no occupancy, but only two of them fit an SM: not used where they would
+        // make between one and two waves of short items (measured at 384 pairs of 408 rows:
+        // 32.8 us against 29.7 us for three splits and the combine; with ~1000-row items the
+        // single launch still wins there).  Requests beyond 2048 rows need the combine anyway;
+        // there the merge on top of it measured as a small loss.
         if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK && env_int("DSA_ITEM_WARPS", 1) != 0) {
-            // Too few pairs to fill the device, and a request fits one (long) row list: the
-            // tensor-core kernel puts kMmaItemWarps warps on one work item and merges them in
-            // shared memory -- the same parallelism without partial results and, up to
-            // kMmaItemWarps pieces, without the combine launch.  Those blocks hold four rings, so
-            // a list of twice the usual length costs no occupancy.  (Longer requests need the
-            // combine anyway; there the merge on top of it measured as a small loss.)
-            pl->mma_kw = kMmaItemWarps;
-            pl->mma_warps = 1;
-            want_split = (want_split + kMmaItemWarps - 1) / kMmaItemWarps;
-            max_chunk = 2 * MAX_CHUNK;
+            const int64_t kw_blocks = pairs * ((want_split + kMmaItemWarps - 1) / kMmaItemWarps);
+            if (kw_blocks <= 2 * kNumSMs || kw_blocks >= 4 * kNumSMs || bound > MAX_CHUNK) {
+                pl->mma_kw = kMmaItemWarps;
+                pl->mma_warps = 1;
+                want_split = (want_split + kMmaItemWarps - 1) / kMmaItemWarps;
+                max_chunk = 2 * MAX_CHUNK;
+            }
         }
         want_split = std::max<int64_t>(want_split, (bound + max_chunk - 1) / max_chunk);
         // Requests too long for one row list are split anyway; when the (request, kv head) pairs
