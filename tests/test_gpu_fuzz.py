@@ -92,3 +92,68 @@ def test_long_single_sequence_many_splits():
         util.assert_close(out, lse, ref, what="long mode %d" % mode)
         idx, cnt = dsa.dsa_debug_kept_indices(prob, diag, inp["max_seq_len"])
         util.assert_kept_equal(idx, cnt, ref, "long mode %d" % mode)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_fused_decode_step(seed):
+    """Random shapes through the fused append + attention call: the current token's rows are taken
+    out of a complete cache (slots poisoned), handed over as k_new / v_new with seq_len one lower,
+    and the oracle's result on the complete cache is expected, with the cache restored bit for bit."""
+    from paper_2609_19702_b200 import binding as dsa
+    from tests.test_gpu_decode_step import _bits, _take_out_current_token
+    rng = np.random.default_rng(9500 + seed)
+    w = _random_case(rng)
+    inp = synth.make_inputs(w, seed=700 + seed)
+    split = int(rng.choice([0, 0, 32, 96]))
+    n_sink = int(rng.choice([0, 0, 2]))
+    hq = w.num_q_heads
+    mh = int(rng.choice(sorted({1, w.num_kv_heads, hq})))
+    trace = synth.random_valid_trace(rng, w.window, w.n_att, (w.batch, mh))
+    cases = [
+        (lambda: None, ora.MODE_DENSE, {}),
+        (lambda: dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra, n_sink=n_sink), ora.MODE_GRID,
+         dict(n_r=w.window, n_att=w.n_att, stride=w.stride, n_sink=n_sink)),
+        (lambda: dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=torch.from_numpy(trace.copy()).cuda(),
+                          n_sink=n_sink), ora.MODE_LIST, dict(n_r=w.window, n_att=w.n_att, trace=trace, n_sink=n_sink)),
+    ]
+    tag = "seed %d: %s split=%d sinks=%d mh=%d" % (seed, w, split, n_sink, mh)
+    for make_diag, mode, kw in cases:
+        ref = util.oracle_run(inp, mode, **kw)
+        prob = dsa.problem_from_host(inp, split_tokens=split)
+        original = (_bits(prob.k_cache).clone(), _bits(prob.v_cache).clone())
+        diag = make_diag()
+        k_new, v_new = _take_out_current_token(prob, inp)
+        out, lse = dsa.alloc_outputs(prob)
+        out.fill_(float("nan"))
+        dsa.dsa_decode_step(prob, diag, k_new, v_new, out, lse, dsa.alloc_workspace(prob, diag))
+        torch.cuda.synchronize()
+        util.assert_close(out, lse, ref, what="%s mode %d" % (tag, mode))
+        assert torch.equal(_bits(prob.k_cache), original[0]) and torch.equal(_bits(prob.v_cache), original[1]), tag
+
+
+def test_two_streams_use_the_library_at_once():
+    """The library keeps no state between calls: two streams with their own problems, outputs and
+    workspaces run interleaved and each gets its own oracle result."""
+    from paper_2609_19702_b200 import binding as dsa
+    jobs = []
+    for i, (index, batch) in enumerate(((5, 3), (4, 2))):
+        w = synth.workload(index, batch=batch)
+        inp = synth.make_inputs(w, seed=40 + i)
+        prob = dsa.problem_from_host(inp)
+        diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+        ref_sparse = util.oracle_run(inp, ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride=w.stride)
+        ref_dense = util.oracle_run(inp, ora.MODE_DENSE)
+        jobs.append(dict(prob=prob, diag=diag, refs=(ref_sparse, ref_dense), stream=torch.cuda.Stream(),
+                         outs=[dsa.alloc_outputs(prob) for _ in range(2)],
+                         ws=(dsa.alloc_workspace(prob, diag), dsa.alloc_workspace(prob, None))))
+    torch.cuda.synchronize()
+    for _ in range(5):                                   # interleave the launches of the two streams
+        for j in jobs:
+            (o_s, l_s), (o_d, l_d) = j["outs"]
+            dsa.dsa_decode_attention_sparse(j["prob"], j["diag"], o_s, l_s, j["ws"][0], stream=j["stream"])
+            dsa.dsa_decode_attention_dense(j["prob"], o_d, l_d, j["ws"][1], stream=j["stream"])
+    torch.cuda.synchronize()
+    for n, j in enumerate(jobs):
+        (o_s, l_s), (o_d, l_d) = j["outs"]
+        util.assert_close(o_s, l_s, j["refs"][0], what="stream %d sparse" % n)
+        util.assert_close(o_d, l_d, j["refs"][1], what="stream %d dense" % n)
