@@ -5,9 +5,10 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <type_traits>
 
-#include "dsa_attn.cuh"
-#include "dsa_attn_mma.cuh"
+#include "dsa_aux.cuh"
+#include "dsa_launch.cuh"
 
 namespace {
 
@@ -21,12 +22,6 @@ int32_t cuda_fail(cudaError_t e) {
 }
 
 constexpr int kNumSMs = 148;
-constexpr int kMaxDevices = 64;
-#ifndef DSA_TUNE_MMA_STAGES
-#define DSA_TUNE_MMA_STAGES 3
-#endif
-constexpr int kMmaItemWarps = 4;                   // warps per work item in small launches
-constexpr int kMmaStages = DSA_TUNE_MMA_STAGES;    // 16-key tiles in flight per warp (+1 being consumed)
 
 int env_int(const char* name, int fallback) {
     const char* v = std::getenv(name);
@@ -34,25 +29,6 @@ int env_int(const char* name, int fallback) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-// Launch `kern` so that it may be scheduled before the kernel queued ahead of it on the stream has
-// finished (programmatic stream serialisation).  Every kernel launched this way starts with
-// griddepcontrol.wait, which holds it until that earlier grid has completed and its writes are
-// visible; after a kernel that never signals early this is an ordinary serialised launch.
-template <class Kern, class... Args>
-cudaError_t launch_pdl(Kern kern, unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, args...);
-}
 
 // The launch plan: how many kept rows one block takes, how many splits that makes.
 struct Plan {
@@ -71,111 +47,25 @@ struct Plan {
     size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
 };
 
-template <typename T, int D, int G, bool HM, bool SEL>
-struct KernelPick {
-    // Small tiles (2 KB of K + 2 KB of V) in a 4-deep ring: 16-20 KB of shared memory per block, so
-    // 8 or more blocks share an SM and their start-up and merge phases overlap each other's
-    // streaming.  (Measured on the paged batch-256 workload: 32-row tiles with 3 blocks/SM reach
-    // 5.7 TB/s, these reach 6.6 TB/s; the dense call is flat at 7.2 TB/s either way.)
-    // -DDSA_TUNE_TILE / -DDSA_TUNE_STAGES override the bf16, head_dim 128 choice in tuning builds.
-    static constexpr int kTileDefault = 2048 / (D * (int)sizeof(T));
-    static constexpr int kStagesDefault = 4;
-#ifdef DSA_TUNE_TILE
-    static constexpr int TILE = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_TILE : kTileDefault;
-#else
-    static constexpr int TILE = kTileDefault;
-#endif
-#ifdef DSA_TUNE_STAGES
-    static constexpr int STAGES = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_STAGES : kStagesDefault;
-#else
-    static constexpr int STAGES = kStagesDefault;
-#endif
-    using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM, SEL>;
-    static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
-    // Tensor-core kernel (bf16 only).  W warps per block share one row list when the mask does not
-    // depend on the head (never with per-head masks or selection).
-    template <int W>
-    static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, kMmaStages, HM, SEL, W>::smem_bytes(chunk, bw); }
-    static size_t smem_mma(int w, int kw, int chunk, int bw) {
-        if (kw > 1) return smem_mma_w<kMmaItemWarps>(chunk, bw);      // one ring per warp either way
-        if constexpr (!HM && !SEL) {
-            if (w == 2) return smem_mma_w<2>(chunk, bw);
-        }
-        return smem_mma_w<1>(chunk, bw);
-    }
-    template <int W, bool APPEND, int KW>
-    static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>;
-        static bool configured[kMaxDevices] = {};
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
-        }
-        return launch_pdl(kern, (unsigned)grid, 32 * W * KW, smem_bytes, st, a);
-    }
-    // `append`: the fused decode step (the kernel reads the current token from a.k_new / a.v_new)
-    template <bool APPEND>
-    static cudaError_t launch_mma_a(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
-                                    cudaStream_t st) {
-        if constexpr (sizeof(T) == 2) {
-            if (kw > 1) return launch_mma_w<1, APPEND, kMmaItemWarps>(a, items, smem_bytes, st);
-            if constexpr (!HM && !SEL) {
-                if (w == 2) return launch_mma_w<2, APPEND, 1>(a, items / 2, smem_bytes, st);
-            }
-            return launch_mma_w<1, APPEND, 1>(a, items, smem_bytes, st);
-        } else {
-            return cudaErrorInvalidValue;
-        }
-    }
-    static cudaError_t launch_mma(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
-                                  cudaStream_t st, bool append) {
-        return append ? launch_mma_a<true>(w, kw, a, items, smem_bytes, st)
-                      : launch_mma_a<false>(w, kw, a, items, smem_bytes, st);
-    }
-    static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
-        static bool configured[kMaxDevices] = {};
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
-        }
-        return launch_pdl(kern, (unsigned)grid, NT, smem_bytes, st, a);
-    }
-};
+// The kernels live in translation units of their own, one per (element type, head_dim): only the
+// declarations of kernel_shape / kernel_launch are visible here, their instantiations are linked in.
 
-// Dispatch over (dtype, head_dim, group size, per-head masks, fused selection).  Selection needs one
-// mask per query head, so it comes with per-head masks whenever the group is larger than one.
+// Dispatch over (dtype, head_dim): f is called with a value of the element type and head_dim as
+// an integral constant.
 template <class F>
-int32_t dispatch(int dtype, int D, int G, bool hm, bool sel, F&& f) {
-#define DSA_CASE_HM(T, DD, GG)                                                         \
-    if (sel) return f(KernelPick<T, DD, GG, (GG > 1), true>{});                        \
-    return hm ? f(KernelPick<T, DD, GG, (GG > 1), false>{}) : f(KernelPick<T, DD, GG, false, false>{});
-#define DSA_CASE_G(T, DD)                         \
-    switch (G) {                                  \
-        case 1: { DSA_CASE_HM(T, DD, 1) }         \
-        case 2: { DSA_CASE_HM(T, DD, 2) }         \
-        case 4: { DSA_CASE_HM(T, DD, 4) }         \
-        case 8: { DSA_CASE_HM(T, DD, 8) }         \
-        default: return DSA_ERR_UNSUPPORTED;      \
-    }
-    if (dtype == DSA_BF16) {
-        if (D == 64) { DSA_CASE_G(__nv_bfloat16, 64) }
-        if (D == 128) { DSA_CASE_G(__nv_bfloat16, 128) }
-    } else if (dtype == DSA_F32) {
-        if (D == 64) { DSA_CASE_G(float, 64) }
-        if (D == 128) { DSA_CASE_G(float, 128) }
-    }
-#undef DSA_CASE_G
-#undef DSA_CASE_HM
+int32_t dispatch(int dtype, int D, F&& f) {
+    if (dtype == DSA_BF16 && D == 64) return f(__nv_bfloat16{}, std::integral_constant<int, 64>{});
+    if (dtype == DSA_BF16 && D == 128) return f(__nv_bfloat16{}, std::integral_constant<int, 128>{});
+    if (dtype == DSA_F32 && D == 64) return f(float{}, std::integral_constant<int, 64>{});
+    if (dtype == DSA_F32 && D == 128) return f(float{}, std::integral_constant<int, 128>{});
     return DSA_ERR_UNSUPPORTED;
+}
+
+KernelQuery kernel_query(const Plan& pl) {
+    KernelQuery q;
+    q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
+    q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw;
+    return q;
 }
 
 // Tokens one request can hold: its logical maximum, or prompt + sinks + ring when bounded.
@@ -260,34 +150,38 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     }
     if (bound < 1) bound = 1;
 
-    size_t smem_probe = 0;
-    rc = dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
-        using P = decltype(pick);
-        pl->tile = P::TILE;
-        pl->stages = P::STAGES;
-        return DSA_OK;
-    });
-    if (rc != DSA_OK) return rc;
     // bf16 runs on the tensor-core kernel (one warp per work item); fp32 on the CUDA-core kernel.
     // DSA_CUDA_CORES=1 forces the latter for bf16 too (comparison runs).
     pl->mma = p->dtype == DSA_BF16 && env_int("DSA_CUDA_CORES", 0) == 0;
     pl->mma_warps = 1;
     pl->mma_kw = 1;
     if (pl->mma) {
-        pl->tile = MMA_KEYS;
-        pl->stages = kMmaStages;
         const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
         // two kv heads per block (measured: 2 beats 1 and 4) when the row list can be shared
         if (shared_mask && p->num_kv_heads % 2 == 0) pl->mma_warps = 2;
     }
+    // tile and ring depth of the kernel that will run (they do not depend on the row-list length)
+    auto shape_of = [&](int chunk, KernelShape* shape) -> int32_t {
+        return dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
+            using T = decltype(t);
+            return kernel_shape<T, decltype(dd)::value>(kernel_query(*pl), chunk, pl->bitmap_words, shape)
+                       ? DSA_OK : DSA_ERR_UNSUPPORTED;
+        });
+    };
+    KernelShape shape = {};
+    rc = shape_of(0, &shape);
+    if (rc != DSA_OK) return rc;
+    pl->tile = shape.tile;
+    pl->stages = shape.stages;
 
     int chunk;
     if (p->split_tokens > 0) {
         chunk = std::min(MAX_CHUNK, round_up(p->split_tokens, pl->tile));
     } else {
-        // One block streams about 12 GB/s on its own, and a split costs the combine launch, so:
-        // split only while fewer than ~4 blocks per SM exist, never below 128 rows per block, and
-        // balance the splits (equal chunks rather than full ones plus a short tail).
+        // One work item streams about 12 GB/s on its own, and a split costs the combine launch, so:
+        // split only while fewer than ~6 warps (4 blocks of the CUDA-core kernel) per SM exist,
+        // never below 96 (128) rows per item, and balance the splits (equal chunks rather than
+        // full ones plus a short tail).
         const int64_t pairs = (int64_t)std::max(p->batch, 1) * p->num_kv_heads;
         const int64_t target = (pl->mma ? 6 : 4) * kNumSMs;        // a work item is a warp / a 4-warp block
         int64_t want_split = std::max<int64_t>(1, (target + pairs - 1) / pairs);
@@ -328,13 +222,9 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->grid = (int64_t)p->batch * p->num_kv_heads * pl->n_split;
     if (pl->grid > 0x7fffffffLL) return DSA_ERR_UNSUPPORTED;
 
-    dispatch(p->dtype, p->head_dim, G, pl->headmask, pl->select, [&](auto pick) -> int32_t {
-        using P = decltype(pick);
-        smem_probe = pl->mma ? P::smem_mma(pl->mma_warps, pl->mma_kw, pl->chunk, pl->bitmap_words)
-                             : P::smem(pl->chunk, pl->bitmap_words);
-        return DSA_OK;
-    });
-    pl->smem = smem_probe;
+    rc = shape_of(pl->chunk, &shape);                         // (the small-launch form may have been chosen since)
+    if (rc != DSA_OK) return rc;
+    pl->smem = shape.smem;
     if (pl->smem > 200 * 1024) return DSA_ERR_UNSUPPORTED;     // window too large for LIST bitmaps
 
     if (pl->n_split > 1) {
@@ -465,10 +355,9 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
         }
     }
     cudaError_t err = cudaSuccess;
-    rc = dispatch(p->dtype, p->head_dim, pl.G, pl.headmask, pl.select, [&](auto pick) -> int32_t {
-        using P = decltype(pick);
-        err = pl.mma ? P::launch_mma(pl.mma_warps, pl.mma_kw, a, pl.grid, pl.smem, st, step && pl.mma)
-                     : P::launch(a, pl.grid, pl.smem, st);
+    rc = dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
+        using T = decltype(t);
+        err = kernel_launch<T, decltype(dd)::value>(kernel_query(pl), step && pl.mma, a, pl.grid, pl.smem, st);
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;

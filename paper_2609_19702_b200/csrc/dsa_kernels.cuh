@@ -1,0 +1,149 @@
+// Kernel selection and launch for one (element type, head_dim): included by the per-type
+// translation units (dsa_kernels_*.cu), which instantiate kernel_shape / kernel_launch.
+#pragma once
+#include "dsa_attn.cuh"
+#include "dsa_attn_mma.cuh"
+#include "dsa_launch.cuh"
+
+namespace dsa {
+
+// Launch `kern` so that it may be scheduled before the kernel queued ahead of it on the stream has
+// finished (programmatic stream serialisation).  Every kernel launched this way starts with
+// griddepcontrol.wait, which holds it until that earlier grid has completed and its writes are
+// visible; after a kernel that never signals early this is an ordinary serialised launch.
+template <class Kern, class... Args>
+cudaError_t launch_pdl(Kern kern, unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+template <typename T, int D, int G, bool HM, bool SEL>
+struct KernelPick {
+    // Small tiles (2 KB of K + 2 KB of V) in a 4-deep ring: 16-20 KB of shared memory per block, so
+    // 8 or more blocks share an SM and their start-up and merge phases overlap each other's
+    // streaming.  (Measured on the paged batch-256 workload: 32-row tiles with 3 blocks/SM reach
+    // 5.7 TB/s, these reach 6.6 TB/s; the dense call is flat at 7.2 TB/s either way.)
+    // -DDSA_TUNE_TILE / -DDSA_TUNE_STAGES override the bf16, head_dim 128 choice in tuning builds.
+    static constexpr int kTileDefault = 2048 / (D * (int)sizeof(T));
+    static constexpr int kStagesDefault = 4;
+#ifdef DSA_TUNE_TILE
+    static constexpr int TILE = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_TILE : kTileDefault;
+#else
+    static constexpr int TILE = kTileDefault;
+#endif
+#ifdef DSA_TUNE_STAGES
+    static constexpr int STAGES = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_STAGES : kStagesDefault;
+#else
+    static constexpr int STAGES = kStagesDefault;
+#endif
+    using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM, SEL>;
+    static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
+    // Tensor-core kernel (bf16 only).  W warps per block share one row list when the mask does not
+    // depend on the head (never with per-head masks or selection).
+    template <int W>
+    static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, kMmaStages, HM, SEL, W>::smem_bytes(chunk, bw); }
+    static size_t smem_mma(int w, int kw, int chunk, int bw) {
+        if (kw > 1) return smem_mma_w<kMmaItemWarps>(chunk, bw);      // one ring per warp either way
+        if constexpr (!HM && !SEL) {
+            if (w == 2) return smem_mma_w<2>(chunk, bw);
+        }
+        return smem_mma_w<1>(chunk, bw);
+    }
+    template <int W, bool APPEND, int KW>
+    static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
+        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>;
+        static bool configured[kMaxDevices] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        }
+        return launch_pdl(kern, (unsigned)grid, 32 * W * KW, smem_bytes, st, a);
+    }
+    // `append`: the fused decode step (the kernel reads the current token from a.k_new / a.v_new)
+    template <bool APPEND>
+    static cudaError_t launch_mma_a(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
+                                    cudaStream_t st) {
+        if constexpr (sizeof(T) == 2) {
+            if (kw > 1) return launch_mma_w<1, APPEND, kMmaItemWarps>(a, items, smem_bytes, st);
+            if constexpr (!HM && !SEL) {
+                if (w == 2) return launch_mma_w<2, APPEND, 1>(a, items / 2, smem_bytes, st);
+            }
+            return launch_mma_w<1, APPEND, 1>(a, items, smem_bytes, st);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
+    static cudaError_t launch_mma(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
+                                  cudaStream_t st, bool append) {
+        return append ? launch_mma_a<true>(w, kw, a, items, smem_bytes, st)
+                      : launch_mma_a<false>(w, kw, a, items, smem_bytes, st);
+    }
+    static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
+        auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
+        static bool configured[kMaxDevices] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        }
+        return launch_pdl(kern, (unsigned)grid, NT, smem_bytes, st, a);
+    }
+};
+
+// Dispatch over (group size, per-head masks, fused selection).  Selection needs one mask per query
+// head, so it comes with per-head masks whenever the group is larger than one.
+template <typename T, int D, class F>
+bool dispatch_variant(const KernelQuery& q, F&& f) {
+#define DSA_CASE_HM(GG)                                                                   \
+    if (q.select) { f(KernelPick<T, D, GG, (GG > 1), true>{}); return true; }             \
+    if (q.headmask) { f(KernelPick<T, D, GG, (GG > 1), false>{}); return true; }          \
+    f(KernelPick<T, D, GG, false, false>{});                                              \
+    return true;
+    switch (q.G) {
+        case 1: { DSA_CASE_HM(1) }
+        case 2: { DSA_CASE_HM(2) }
+        case 4: { DSA_CASE_HM(4) }
+        case 8: { DSA_CASE_HM(8) }
+        default: return false;
+    }
+#undef DSA_CASE_HM
+}
+
+template <typename T, int D>
+bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape* out) {
+    return dispatch_variant<T, D>(q, [&](auto pick) {
+        using P = decltype(pick);
+        out->tile = q.mma ? MMA_KEYS : P::TILE;
+        out->stages = q.mma ? kMmaStages : P::STAGES;
+        out->smem = q.mma ? P::smem_mma(q.mma_warps, q.mma_kw, chunk, bitmap_words) : P::smem(chunk, bitmap_words);
+    });
+}
+
+template <typename T, int D>
+cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
+                          cudaStream_t st) {
+    cudaError_t err = cudaErrorInvalidValue;
+    dispatch_variant<T, D>(q, [&](auto pick) {
+        using P = decltype(pick);
+        err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, a, items, smem, st, append) : P::launch(a, items, smem, st);
+    });
+    return err;
+}
+
+}  // namespace dsa

@@ -1,0 +1,7 @@
+// Attention kernels for bf16 caches with head_dim 64 (see dsa_launch.cuh).
+#include "dsa_kernels.cuh"
+
+namespace dsa {
+template bool kernel_shape<__nv_bfloat16, 64>(const KernelQuery&, int, int, KernelShape*);
+template cudaError_t kernel_launch<__nv_bfloat16, 64>(const KernelQuery&, bool, const AttnArgs&, int64_t, size_t, cudaStream_t);
+}  // namespace dsa

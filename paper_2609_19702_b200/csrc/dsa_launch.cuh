@@ -1,0 +1,42 @@
+// The seam between the host-side planner (dsa_api.cu) and the attention kernels: the kernels of
+// each (element type, head_dim) are instantiated in a translation unit of their own, so that the
+// library builds in parallel, and are reached through the two function templates declared here.
+#pragma once
+#include "dsa_common.cuh"
+
+namespace dsa {
+
+constexpr int kMaxDevices = 64;
+constexpr int kMmaItemWarps = 4;                   // warps per work item in small launches
+#ifndef DSA_TUNE_MMA_STAGES
+#define DSA_TUNE_MMA_STAGES 3
+#endif
+constexpr int kMmaStages = DSA_TUNE_MMA_STAGES;    // 16-key tiles in flight per warp (+1 being consumed)
+
+// Which kernel variant a call needs.
+struct KernelQuery {
+    int G;                   // query heads per kv head: 1, 2, 4 or 8
+    bool headmask;           // one mask per query head inside a group
+    bool select;             // fused phase-2 selection
+    bool mma;                // tensor-core kernel (bf16) rather than the CUDA-core kernel
+    int mma_warps;           // tensor-core kernel: kv heads per block that share one row list (1 or 2)
+    int mma_kw;              // tensor-core kernel: warps that share one work item (1 or kMmaItemWarps)
+};
+
+struct KernelShape {
+    int tile;                // keys per staged tile
+    int stages;              // tiles in flight (per warp for the tensor-core kernel)
+    size_t smem;             // dynamic shared memory per block for a row list of `chunk` rows
+};
+
+// Shape of the variant `q` of element type T and head_dim D.  Returns false for an unsupported G.
+template <typename T, int D>
+bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape* out);
+
+// Launch it: `items` (request, kv head, split) work items; `append`: the fused decode step (the
+// kernel reads the current token's rows from a.k_new / a.v_new and stores them to the cache).
+template <typename T, int D>
+cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
+                          cudaStream_t st);
+
+}  // namespace dsa
