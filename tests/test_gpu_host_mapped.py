@@ -67,6 +67,14 @@ def test_host_mapped_step_matches_oracle_and_device_call(dsa, index, batch, mode
         assert torch.equal(h["out"].view(torch.int16), ref_out.cpu().view(torch.int16))
         assert torch.equal(h["lse"], ref_lse.cpu())
     assert torch.equal(prob.seq_len.cpu(), h["seq"])
+    # the host rewrites its buffers between steps: the next call must see the new q (here: -q)
+    flipped = dict(inp, q=inp["q"] ^ np.uint16(0x8000))
+    h["q"].view(torch.int16).copy_(torch.from_numpy(flipped["q"].view(np.int16)))
+    ref2 = (util.oracle_run(flipped, ora.MODE_DENSE) if diag is None else
+            util.oracle_run(flipped, ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride=w.stride))
+    dsa.dsa_decode_attention_host_mapped(prob, diag, h["q"], h["seq"], h["pl"], h["bt"], h["out"], h["lse"], ws)
+    torch.cuda.synchronize()
+    util.assert_close(h["out"], h["lse"], ref2, what="host-mapped %s config %d, rewritten q" % (mode, index))
     if n_split == 1:
         assert torch.equal(prob.q, q_before), "q is read from the host buffer: the device copy stays untouched"
     else:
