@@ -29,11 +29,29 @@ def _random_case(rng):
                           positional=bool(rng.integers(0, 2)), paged=paged, block_size=bs)
 
 
-@pytest.mark.parametrize("seed", range(24))
+def _random_large_case(rng):
+    """Up to 3000 image tokens and windows up to 1500: several tiles per warp, several splits,
+    the four-warps-per-item plans, long row lists."""
+    g = int(rng.choice([1, 2, 4, 8]))
+    hkv = int(rng.choice([1, 2, 4, 8]))
+    d = int(rng.choice([64, 128]))
+    grid_w = int(rng.integers(8, 70))
+    extra = int(rng.integers(0, 2))
+    grid_h = int(rng.integers(8, max(9, 3000 // (grid_w + extra))))
+    n_img = grid_h * (grid_w + extra)
+    n_r = int(rng.integers(64, min(n_img, 1500) + 1))
+    n_att = int(rng.integers(1, n_r + 1))
+    l_p = int(rng.choice([0, 33, 200, 700]))
+    return synth.Workload("fuzzbig", 0, int(rng.integers(1, 9)), g * hkv, hkv, d, l_p, grid_h, grid_w, extra, n_r,
+                          n_att, 1, n_img, positional=bool(rng.integers(0, 2)), paged=bool(rng.integers(0, 2)),
+                          block_size=int(rng.choice([4, 16, 64])))
+
+
+@pytest.mark.parametrize("seed", list(range(24)) + list(range(1000, 1010)))
 def test_random_problem(seed):
     from paper_2609_19702_b200 import binding as dsa
     rng = np.random.default_rng(9000 + seed)
-    w = _random_case(rng)
+    w = _random_case(rng) if seed < 1000 else _random_large_case(rng)
     inp = synth.make_inputs(w, seed=500 + seed)
     f32 = bool(rng.integers(0, 4) == 0)
     split = int(rng.choice([0, 0, 16, 48, 130]))
@@ -94,7 +112,7 @@ def test_long_single_sequence_many_splits():
         util.assert_kept_equal(idx, cnt, ref, "long mode %d" % mode)
 
 
-@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("seed", list(range(12)) + list(range(2000, 2006)))
 def test_random_fused_decode_step(seed):
     """Random shapes through the fused append + attention call: the current token's rows are taken
     out of a complete cache (slots poisoned), handed over as k_new / v_new with seq_len one lower,
@@ -102,7 +120,7 @@ def test_random_fused_decode_step(seed):
     from paper_2609_19702_b200 import binding as dsa
     from tests.test_gpu_decode_step import _bits, _take_out_current_token
     rng = np.random.default_rng(9500 + seed)
-    w = _random_case(rng)
+    w = _random_case(rng) if seed < 1000 else _random_large_case(rng)
     inp = synth.make_inputs(w, seed=700 + seed)
     split = int(rng.choice([0, 0, 32, 96]))
     n_sink = int(rng.choice([0, 0, 2]))
