@@ -22,8 +22,9 @@
  *   - Return value: DSA_OK or a negative dsa_status.  After DSA_ERR_CUDA the CUDA error code is
  *     available from dsa_last_cuda_error().
  *   - The first launch of each kernel variant on a device also configures it (a one-time
- *     attribute call); make the first call of a given shape outside any stream capture.  After
- *     that the attention, combine and append calls can be captured into CUDA graphs.
+ *     attribute call that must not happen inside a stream capture): call dsa_prepare() once per
+ *     device, or make the first call of a given shape, before capturing.  After that every call
+ *     of this header can be captured into CUDA graphs.
  *   - There is no CPU path: without a CUDA device every compute call fails with DSA_ERR_CUDA.
  *
  * Positions.  For request b, prompt_len[b] = L_p tokens of prompt come first in the cache and
@@ -188,6 +189,14 @@ DSA_API int32_t dsa_version(void);
 DSA_API const char *dsa_status_string(int32_t status);
 /* CUDA error code recorded by the last failing call of this thread (0 if none). */
 DSA_API int32_t dsa_last_cuda_error(void);
+
+/*
+ * Configure every kernel variant of the library for the CURRENT device (a few hundred one-time
+ * attribute calls, no launch, no allocation).  Optional: calls do it lazily for the variant they
+ * need; required only before a stream capture whose calls would otherwise be the first of their
+ * shape on this device.
+ */
+DSA_API int32_t dsa_prepare(void);
 
 /* Bytes of workspace the attention calls need for `problem` (diag == NULL: dense call). */
 DSA_API int32_t dsa_workspace_size(const dsa_problem *problem, const dsa_diag_params *diag, size_t *bytes);

@@ -24,7 +24,7 @@ EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_works
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
            "dsa_combine_splits", "dsa_debug_kept_indices",
            "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
-           "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len"]
+           "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len", "dsa_prepare"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -82,6 +82,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
     lib.dsa_decode_attention_host_io.restype = i32
     lib.dsa_decode_attention_host_io.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.dsa_prepare.restype = i32
+    lib.dsa_prepare.argtypes = []
     lib.dsa_decode_step.restype = i32
     lib.dsa_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_advance_seq_len.restype = i32
@@ -214,6 +216,12 @@ def dsa_workspace_size(problem: Problem, diag: Optional[Diag] = None) -> int:
     n = ctypes.c_size_t(0)
     _check("dsa_workspace_size", _lib.dsa_workspace_size(_ref(p), _ref(d), ctypes.byref(n)))
     return int(n.value)
+
+
+def dsa_prepare() -> None:
+    """Configure every kernel variant for the current CUDA device (needed only before capturing
+    calls that would otherwise be the first of their shape on this device)."""
+    _check("dsa_prepare", _lib.dsa_prepare())
 
 
 def dsa_query_plan(problem: Problem, diag: Optional[Diag] = None) -> dsa_plan_info:

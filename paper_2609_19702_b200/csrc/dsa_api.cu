@@ -409,6 +409,14 @@ const char* dsa_status_string(int32_t status) {
 
 int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
 
+int32_t dsa_prepare(void) {
+    cudaError_t e = kernel_prepare<__nv_bfloat16, 64>();
+    if (e == cudaSuccess) e = kernel_prepare<__nv_bfloat16, 128>();
+    if (e == cudaSuccess) e = kernel_prepare<float, 64>();
+    if (e == cudaSuccess) e = kernel_prepare<float, 128>();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+}
+
 int32_t dsa_workspace_size(const dsa_problem* problem, const dsa_diag_params* diag, size_t* bytes) {
     if (!bytes) return DSA_ERR_INVALID_ARG;
     Plan pl;

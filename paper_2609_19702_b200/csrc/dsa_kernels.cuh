@@ -5,6 +5,8 @@
 #include "dsa_attn_mma.cuh"
 #include "dsa_launch.cuh"
 
+#include <type_traits>
+
 namespace dsa {
 
 // Launch `kern` so that it may be scheduled before the kernel queued ahead of it on the stream has
@@ -58,19 +60,54 @@ struct KernelPick {
         }
         return smem_mma_w<1>(chunk, bw);
     }
-    template <int W, bool APPEND, int KW>
-    static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>;
-        static bool configured[kMaxDevices] = {};
+    // Kernels that use more than 48 KB of dynamic shared memory must be told so once per device.
+    template <class Kern>
+    static cudaError_t ensure_configured(Kern kern, bool* done /* [kMaxDevices] */) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+        if (dev < 0 || dev >= kMaxDevices || !done[dev]) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
             if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+            if (dev >= 0 && dev < kMaxDevices) done[dev] = true;
         }
+        return cudaSuccess;
+    }
+    template <int W, bool APPEND, int KW>
+    static bool* mma_configured() { static bool done[kMaxDevices] = {}; return done; }
+    static bool* cc_configured() { static bool done[kMaxDevices] = {}; return done; }
+
+    template <int W, bool APPEND, int KW>
+    static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
+        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>;
+        const cudaError_t e = ensure_configured(kern, mma_configured<W, APPEND, KW>());
+        if (e != cudaSuccess) return e;
         return launch_pdl(kern, (unsigned)grid, 32 * W * KW, smem_bytes, st, a);
+    }
+    // Configure every kernel of this variant for the current device (see dsa_prepare).
+    static cudaError_t prepare() {
+        cudaError_t e = ensure_configured(dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>, cc_configured());
+        if constexpr (sizeof(T) == 2) {
+            auto mma = [&](auto w, auto app, auto kw) {
+                constexpr int W = decltype(w)::value, KW = decltype(kw)::value;
+                constexpr bool APPEND = decltype(app)::value;
+                if (e == cudaSuccess)
+                    e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>,
+                                          mma_configured<W, APPEND, KW>());
+            };
+            using one = std::integral_constant<int, 1>;
+            using two = std::integral_constant<int, 2>;
+            using four = std::integral_constant<int, kMmaItemWarps>;
+            mma(one{}, std::false_type{}, one{});
+            mma(one{}, std::true_type{}, one{});
+            mma(one{}, std::false_type{}, four{});
+            mma(one{}, std::true_type{}, four{});
+            if constexpr (!HM && !SEL) {
+                mma(two{}, std::false_type{}, one{});
+                mma(two{}, std::true_type{}, one{});
+            }
+        }
+        return e;
     }
     // `append`: the fused decode step (the kernel reads the current token from a.k_new / a.v_new)
     template <bool APPEND>
@@ -93,15 +130,8 @@ struct KernelPick {
     }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
         auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
-        static bool configured[kMaxDevices] = {};
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
+        const cudaError_t e = ensure_configured(kern, cc_configured());
         if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
-        }
         return launch_pdl(kern, (unsigned)grid, NT, smem_bytes, st, a);
     }
 };
@@ -144,6 +174,20 @@ cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, 
         err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, a, items, smem, st, append) : P::launch(a, items, smem, st);
     });
     return err;
+}
+
+template <typename T, int D>
+cudaError_t kernel_prepare() {
+    cudaError_t e = cudaSuccess;
+    for (int g = 1; g <= 8 && e == cudaSuccess; g *= 2) {
+        for (int variant = 0; variant < 3 && e == cudaSuccess; ++variant) {
+            KernelQuery q = {};
+            q.G = g; q.headmask = variant >= 1; q.select = variant == 2;
+            if (g == 1 && variant == 1) continue;           // (a group of one has no per-head variant of its own)
+            dispatch_variant<T, D>(q, [&](auto pick) { e = decltype(pick)::prepare(); });
+        }
+    }
+    return e;
 }
 
 }  // namespace dsa

@@ -39,4 +39,9 @@ template <typename T, int D>
 cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
                           cudaStream_t st);
 
+// Configure every variant of (T, D) for the current device, so that no later launch has to (a
+// launch inside a stream capture must not).
+template <typename T, int D>
+cudaError_t kernel_prepare();
+
 }  // namespace dsa
