@@ -42,6 +42,7 @@ struct Plan {
     bool mma;            // bf16: one warp per work item, tensor-core tiles
     int mma_warps;       // warps (= kv heads) per block that share one row list
     int mma_kw;          // warps that share one work item (small launches), 1 or kMmaItemWarps
+    int mma_stages;      // ring depth of the tensor-core kernel
     int64_t grid;
     size_t smem;
     size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
@@ -64,7 +65,7 @@ int32_t dispatch(int dtype, int D, F&& f) {
 KernelQuery kernel_query(const Plan& pl) {
     KernelQuery q;
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
-    q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw;
+    q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
     return q;
 }
 
@@ -155,6 +156,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->mma = p->dtype == DSA_BF16 && env_int("DSA_CUDA_CORES", 0) == 0;
     pl->mma_warps = 1;
     pl->mma_kw = 1;
+    pl->mma_stages = kMmaStages;
     if (pl->mma) {
         const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
         // two kv heads per block (measured: 2 beats 1 and 4) when the row list can be shared
@@ -224,6 +226,49 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
 
     rc = shape_of(pl->chunk, &shape);                         // (the small-launch form may have been chosen since)
     if (rc != DSA_OK) return rc;
+    // Ring depth of the two-heads-per-block kernel.  Shared memory decides how many blocks an SM
+    // holds, and a launch of a few waves pays for every block beyond a whole number of them: a
+    // last wave costs at least about half a full one, however few blocks it has (measured on the
+    // paged workload, 32 heads: batch 36 -> 40 with the deep ring 43 -> 64 us).  The shallow ring
+    // fits half as many blocks again per SM (and loses about 1 % when waves are many), so estimate
+    // both and take the shallow one when it is clearly cheaper (batch 40 / 48 / 80: 48 / 55 / 94 us shallow against 64 / 67 / 102 deep;
+    // batch 64 / 72: 73 / 79 deep against 88 / 91 shallow).
+    // Only for unsplit plans: the splits of a long request differ so much in length (many are
+    // empty) that their blocks pack into waves far better than the estimate assumes (measured: a
+    // loss of 10 % on the dense calls at batch 1-8).
+    if (pl->mma && pl->mma_warps == 2 && pl->mma_kw == 1 && p->split_tokens == 0 &&
+        (pl->n_split == 1 || env_int("DSA_MMA_STAGES", 0) == kMmaStagesShallow) &&
+        env_int("DSA_MMA_STAGES", 0) != kMmaStages) {
+        Plan alt = *pl;
+        alt.mma_stages = kMmaStagesShallow;
+        KernelShape shallow = {};
+        const int32_t rc2 = dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
+            using T = decltype(t);
+            return kernel_shape<T, decltype(dd)::value>(kernel_query(alt), pl->chunk, pl->bitmap_words, &shallow)
+                       ? DSA_OK : DSA_ERR_UNSUPPORTED;
+        });
+        auto cost = [&](size_t smem) {
+            // blocks an SM holds: shared memory (1 KB of it reserved per block), at most 8 by registers
+            const int64_t per_sm = std::min<int64_t>(8, (int64_t)(227 * 1024) / (int64_t)(smem + 1024));
+            const double cap = (double)std::max<int64_t>(per_sm, 1) * kNumSMs;
+            const double waves = (double)(pl->grid / 2) / cap;
+            double whole = std::floor(waves), rest = waves - whole;
+            if (rest < 0.05) rest = 0;                        // a few extra blocks ride on the shortest items
+            if (rest > 0 && whole >= 1) rest = std::max(rest, 0.47);
+            return (whole + rest) * cap;
+        };
+        if (rc2 == DSA_OK && shallow.stages == kMmaStagesShallow) {
+            const bool forced = env_int("DSA_MMA_STAGES", 0) == kMmaStagesShallow;
+            // (with many waves the two are within a few per cent either way: stay with the deep ring
+            // unless the estimate is clearly better)
+            const double margin = (double)(pl->grid / 2) < 3.0 * 4 * kNumSMs ? 1.0 : 0.97;
+            if (forced || cost(shallow.smem) < margin * cost(shape.smem)) {
+                pl->mma_stages = kMmaStagesShallow;
+                pl->stages = shallow.stages;
+                shape = shallow;
+            }
+        }
+    }
     pl->smem = shape.smem;
     if (pl->smem > 200 * 1024) return DSA_ERR_UNSUPPORTED;     // window too large for LIST bitmaps
 

@@ -51,12 +51,15 @@ struct KernelPick {
     static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
     // Tensor-core kernel (bf16 only).  W warps per block share one row list when the mask does not
     // depend on the head (never with per-head masks or selection).
-    template <int W>
-    static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, kMmaStages, HM, SEL, W>::smem_bytes(chunk, bw); }
-    static size_t smem_mma(int w, int kw, int chunk, int bw) {
+    // The two-heads-per-block form also exists with a shallower ring (kMmaStagesShallow): more
+    // blocks per SM, for launches that would otherwise spill a little into another wave.
+    template <int W, int ST = kMmaStages>
+    static size_t smem_mma_w(int chunk, int bw) { return MmaCfg<D, G, ST, HM, SEL, W>::smem_bytes(chunk, bw); }
+    static size_t smem_mma(int w, int kw, int stages, int chunk, int bw) {
         if (kw > 1) return smem_mma_w<kMmaItemWarps>(chunk, bw);      // one ring per warp either way
         if constexpr (!HM && !SEL) {
-            if (w == 2) return smem_mma_w<2>(chunk, bw);
+            if (w == 2) return stages == kMmaStagesShallow ? smem_mma_w<2, kMmaStagesShallow>(chunk, bw)
+                                                           : smem_mma_w<2>(chunk, bw);
         }
         return smem_mma_w<1>(chunk, bw);
     }
@@ -73,14 +76,14 @@ struct KernelPick {
         }
         return cudaSuccess;
     }
-    template <int W, bool APPEND, int KW>
+    template <int W, bool APPEND, int KW, int ST>
     static bool* mma_configured() { static bool done[kMaxDevices] = {}; return done; }
     static bool* cc_configured() { static bool done[kMaxDevices] = {}; return done; }
 
-    template <int W, bool APPEND, int KW>
+    template <int W, bool APPEND, int KW, int ST = kMmaStages>
     static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
-        auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>;
-        const cudaError_t e = ensure_configured(kern, mma_configured<W, APPEND, KW>());
+        auto kern = dsa_attn_mma_kernel<D, G, ST, HM, SEL, W, APPEND, KW>;
+        const cudaError_t e = ensure_configured(kern, mma_configured<W, APPEND, KW, ST>());
         if (e != cudaSuccess) return e;
         return launch_pdl(kern, (unsigned)grid, 32 * W * KW, smem_bytes, st, a);
     }
@@ -88,34 +91,40 @@ struct KernelPick {
     static cudaError_t prepare() {
         cudaError_t e = ensure_configured(dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>, cc_configured());
         if constexpr (sizeof(T) == 2) {
-            auto mma = [&](auto w, auto app, auto kw) {
-                constexpr int W = decltype(w)::value, KW = decltype(kw)::value;
+            auto mma = [&](auto w, auto app, auto kw, auto stg) {
+                constexpr int W = decltype(w)::value, KW = decltype(kw)::value, ST = decltype(stg)::value;
                 constexpr bool APPEND = decltype(app)::value;
                 if (e == cudaSuccess)
-                    e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, W, APPEND, KW>,
-                                          mma_configured<W, APPEND, KW>());
+                    e = ensure_configured(dsa_attn_mma_kernel<D, G, ST, HM, SEL, W, APPEND, KW>,
+                                          mma_configured<W, APPEND, KW, ST>());
             };
             using one = std::integral_constant<int, 1>;
             using two = std::integral_constant<int, 2>;
             using four = std::integral_constant<int, kMmaItemWarps>;
-            mma(one{}, std::false_type{}, one{});
-            mma(one{}, std::true_type{}, one{});
-            mma(one{}, std::false_type{}, four{});
-            mma(one{}, std::true_type{}, four{});
+            using deep = std::integral_constant<int, kMmaStages>;
+            using shallow = std::integral_constant<int, kMmaStagesShallow>;
+            mma(one{}, std::false_type{}, one{}, deep{});
+            mma(one{}, std::true_type{}, one{}, deep{});
+            mma(one{}, std::false_type{}, four{}, deep{});
+            mma(one{}, std::true_type{}, four{}, deep{});
             if constexpr (!HM && !SEL) {
-                mma(two{}, std::false_type{}, one{});
-                mma(two{}, std::true_type{}, one{});
+                mma(two{}, std::false_type{}, one{}, deep{});
+                mma(two{}, std::true_type{}, one{}, deep{});
+                mma(two{}, std::false_type{}, one{}, shallow{});
+                mma(two{}, std::true_type{}, one{}, shallow{});
             }
         }
         return e;
     }
     // `append`: the fused decode step (the kernel reads the current token from a.k_new / a.v_new)
     template <bool APPEND>
-    static cudaError_t launch_mma_a(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
+    static cudaError_t launch_mma_a(int w, int kw, int stages, const AttnArgs& a, int64_t items, size_t smem_bytes,
                                     cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
             if (kw > 1) return launch_mma_w<1, APPEND, kMmaItemWarps>(a, items, smem_bytes, st);
             if constexpr (!HM && !SEL) {
+                if (w == 2 && stages == kMmaStagesShallow)
+                    return launch_mma_w<2, APPEND, 1, kMmaStagesShallow>(a, items / 2, smem_bytes, st);
                 if (w == 2) return launch_mma_w<2, APPEND, 1>(a, items / 2, smem_bytes, st);
             }
             return launch_mma_w<1, APPEND, 1>(a, items, smem_bytes, st);
@@ -123,10 +132,10 @@ struct KernelPick {
             return cudaErrorInvalidValue;
         }
     }
-    static cudaError_t launch_mma(int w, int kw, const AttnArgs& a, int64_t items, size_t smem_bytes,
+    static cudaError_t launch_mma(int w, int kw, int stages, const AttnArgs& a, int64_t items, size_t smem_bytes,
                                   cudaStream_t st, bool append) {
-        return append ? launch_mma_a<true>(w, kw, a, items, smem_bytes, st)
-                      : launch_mma_a<false>(w, kw, a, items, smem_bytes, st);
+        return append ? launch_mma_a<true>(w, kw, stages, a, items, smem_bytes, st)
+                      : launch_mma_a<false>(w, kw, stages, a, items, smem_bytes, st);
     }
     static cudaError_t launch(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {
         auto kern = dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>;
@@ -160,8 +169,11 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
     return dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
         out->tile = q.mma ? MMA_KEYS : P::TILE;
-        out->stages = q.mma ? kMmaStages : P::STAGES;
-        out->smem = q.mma ? P::smem_mma(q.mma_warps, q.mma_kw, chunk, bitmap_words) : P::smem(chunk, bitmap_words);
+        const bool shallow = q.mma && q.mma_stages == kMmaStagesShallow && q.mma_warps == 2 && q.mma_kw == 1 &&
+                             !q.headmask && !q.select;
+        out->stages = q.mma ? (shallow ? kMmaStagesShallow : kMmaStages) : P::STAGES;
+        out->smem = q.mma ? P::smem_mma(q.mma_warps, q.mma_kw, out->stages, chunk, bitmap_words)
+                          : P::smem(chunk, bitmap_words);
     });
 }
 
@@ -171,7 +183,8 @@ cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, 
     cudaError_t err = cudaErrorInvalidValue;
     dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
-        err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, a, items, smem, st, append) : P::launch(a, items, smem, st);
+        err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, q.mma_stages, a, items, smem, st, append)
+                    : P::launch(a, items, smem, st);
     });
     return err;
 }

@@ -12,6 +12,7 @@ constexpr int kMmaItemWarps = 4;                   // warps per work item in sma
 #define DSA_TUNE_MMA_STAGES 3
 #endif
 constexpr int kMmaStages = DSA_TUNE_MMA_STAGES;    // 16-key tiles in flight per warp (+1 being consumed)
+constexpr int kMmaStagesShallow = 2;               // the shallow-ring form of the two-heads-per-block kernel
 
 // Which kernel variant a call needs.
 struct KernelQuery {
@@ -21,6 +22,7 @@ struct KernelQuery {
     bool mma;                // tensor-core kernel (bf16) rather than the CUDA-core kernel
     int mma_warps;           // tensor-core kernel: kv heads per block that share one row list (1 or 2)
     int mma_kw;              // tensor-core kernel: warps that share one work item (1 or kMmaItemWarps)
+    int mma_stages;          // tensor-core kernel: kMmaStages, or kMmaStagesShallow (two heads per block only)
 };
 
 struct KernelShape {

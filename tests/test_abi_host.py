@@ -166,3 +166,20 @@ def test_newer_entry_points_validate_before_touching_a_device(dsa):
     host_io = lib.dsa_decode_attention_host_io
     host_io.argtypes = [ctypes.c_void_p] * 11 + [ctypes.c_size_t, ctypes.c_void_p]
     assert host_io(ctypes.byref(p), ctypes.byref(d), None, hp, hp, None, fake, fake, hp, hp, None, 0, None) == -1
+
+
+def test_ring_depth_follows_the_wave_estimate(dsa):
+    def stages(batch):
+        rc, info = _plan(dsa, _problem(dsa, batch=batch, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,
+                                       max_prompt_len=200), _diag(dsa, window=512, n_att=208, grid_w=64))
+        assert rc == 0 and info.n_split == 1 and info.item_warps == 1
+        return info.stages
+    # 592 two-head blocks fit at once with the deep ring, 888 with the shallow one
+    assert stages(36) == 3          # 576 blocks: one wave either way
+    assert stages(40) == 2          # 640: a second wave of 48 blocks, or one shallow wave
+    assert stages(48) == 2
+    assert stages(64) == 3          # 1024: two waves either way, the deep ones are shorter
+    assert stages(256) == 3         # many waves: no difference worth the shallower pipeline
+    # split plans keep the deep ring
+    rc, info = _plan(dsa, _problem(dsa, batch=8, num_q_heads=32, num_kv_heads=32, max_seq_len=4360))
+    assert rc == 0 and info.n_split > 1 and info.stages == 3

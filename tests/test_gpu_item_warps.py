@@ -101,3 +101,27 @@ def test_shared_item_path_agrees_with_one_warp_per_item(dsa, name, make, splits)
         if t1 is not None:
             # the selected distances (one new trace entry per head) must be the same keys
             assert torch.equal(t1.cpu(), t0.cpu())
+
+
+def test_shallow_ring_form_matches_the_oracle(dsa):
+    """The two-heads-per-block kernel with a two-stage ring: chosen by the planner when the deep
+    ring would spill a few blocks into another wave, and forced here on the standard cases."""
+    # 40 requests x 32 kv heads = 640 blocks: 1.08 waves with the deep ring, 0.72 with the shallow one
+    w = synth.Workload("shallow", 95, 40, 32, 32, 128, 20, 10, 10, 0, 64, 20, 1, 100)
+    inp = synth.make_inputs(w)
+    grid = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    plan = _plan(dsa, inp, grid)
+    assert plan.stages == 2 and plan.item_warps == 1 and plan.n_split == 1
+    _check_all_modes(dsa, inp, list_heads=(1,), seed=5, what="shallow ring, chosen")
+    os.environ["DSA_MMA_STAGES"] = "2"
+    try:
+        for make in (lambda: synth.workload(5, batch=3), lambda: synth.workload(2, batch=8)):
+            w2 = make()
+            inp2 = synth.make_inputs(w2)
+            prob = dsa.problem_from_host(inp2, split_tokens=0)
+            g2 = dsa.Diag(dsa.DSA_MASK_GRID, w2.window, w2.n_att, w2.grid_w, w2.row_extra)
+            if w2.num_kv_heads % 2 == 0 and dsa.dsa_query_plan(prob, g2).item_warps == 1:
+                assert dsa.dsa_query_plan(prob, g2).stages == 2
+            _check_all_modes(dsa, inp2, list_heads=(1,), seed=6, what="shallow ring, forced")
+    finally:
+        os.environ.pop("DSA_MMA_STAGES", None)
