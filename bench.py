@@ -516,7 +516,7 @@ def run_ours(args):
     # ---- variants: dense and the other window, same library, same batch --------------------
     variants = {}
     if not args.no_variants and args.mode == "sparse":
-        vsteps = max(5, args.steps // 10)
+        vsteps = max(5, args.steps // 4)
         todo = [("dense", w)]
         if w.index == 5:
             todo.append(("sparse", synth.workload(5, batch=w.batch, window=1024, n_att=416)))
