@@ -54,3 +54,16 @@ def test_config5_batch256_sampled_requests():
         # property that holds for every request: kept count = prompt + min(p, N_att) (or p)
         want = w.prompt_len + (pos if diag is None else np.minimum(pos, diag.n_att))
         assert np.array_equal(cnt.cpu().numpy()[:, 0], want)
+    # the end-to-end call of the benchmark at this size (step inputs and results in pinned host
+    # memory): bit for bit what the device-buffer call gives
+    diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 208, w.grid_w, w.row_extra)
+    ws = dsa.alloc_workspace(prob, diag)
+    dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+    torch.cuda.synchronize()
+    h_q, h_seq, h_pl = prob.q.cpu().pin_memory(), prob.seq_len.cpu().pin_memory(), prob.prompt_len.cpu().pin_memory()
+    h_bt = prob.block_table.cpu().pin_memory()
+    h_out = torch.full(out.shape, float("nan"), dtype=out.dtype).pin_memory()
+    h_lse = torch.full(lse.shape, float("nan"), dtype=lse.dtype).pin_memory()
+    dsa.dsa_decode_attention_host_mapped(prob, diag, h_q, h_seq, h_pl, h_bt, h_out, h_lse, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(h_out.view(torch.int16), out.cpu().view(torch.int16)) and torch.equal(h_lse, lse.cpu())
