@@ -617,7 +617,8 @@ def run_ours(args):
                        "plan": {"split_tokens": plan.split_tokens, "n_split": plan.n_split,
                                 "grid_blocks": plan.grid_blocks, "smem_bytes": plan.smem_bytes,
                                 "tile_tokens": plan.tile_tokens, "stages": plan.stages,
-                                "tensor_cores": plan.tensor_cores, "work_items": plan.work_items}},
+                                "tensor_cores": plan.tensor_cores, "work_items": plan.work_items,
+                                "item_warps": plan.item_warps}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }
