@@ -53,12 +53,16 @@ def _near_tie(w, q, k, t, h, o_gpu, o_ref):
     return abs(lg - lr) <= 1e-4 * max(1.0, abs(lr))
 
 
-@pytest.mark.parametrize("hq,hkv,d,split,n_sink", [(8, 8, 64, 0, 0), (8, 2, 128, 0, 0), (4, 4, 128, 16, 0),
-                                                 (8, 4, 64, 24, 2)])
-def test_every_step_of_one_sequence(dsa, hq, hkv, d, split, n_sink):
+@pytest.mark.parametrize("hq,hkv,d,split,n_sink,positional", [
+    (8, 8, 64, 0, 0, False), (8, 2, 128, 0, 0, False), (4, 4, 128, 16, 0, False), (8, 4, 64, 24, 2, False),
+    (8, 8, 64, 0, 0, True), (8, 2, 128, 16, 0, True)])
+def test_every_step_of_one_sequence(dsa, hq, hkv, d, split, n_sink, positional):
     # 16x16 grid like the tiny configuration: one call holds every decode step of the sequence,
-    # each request with the oracle's trace up to its own step
-    w = synth.Workload("sel", 61, 256, hq, hkv, d, 32, 16, 16, 0, 64, 13, 1, 256, share_cache=True)
+    # each request with the oracle's trace up to its own step.  With the positional component in
+    # q and k, tokens of the same image column score higher, so the selection is no longer a
+    # draw among equals.
+    w = synth.Workload("sel", 61, 256, hq, hkv, d, 32, 16, 16, 0, 64, 13, 1, 256, share_cache=True,
+                       positional=positional)
     inp = synth.make_inputs(w)
     q, k = _trajectory(w, inp)
     traces = _oracle_traces(w, inp, n_sink)
