@@ -312,6 +312,38 @@ def selection_overhead(torch, dsa, synth, dev):
     return res
 
 
+def mask_variants(torch, dsa, synth, dev, peak):
+    """The mask variants of the paper's comparison at one attention budget (Section 5: sliding
+    window, StreamingLLM, diagonal, diagonal + 4 sinks; here N_att = 208 of window 512 on the paged
+    batch-256 workload), from the same kernel: time and bandwidth on the rows each one keeps."""
+    w = synth.workload(5, batch=256)
+    inputs = synth.make_inputs_device(w, dev)
+    prob = dsa.Problem(
+        q=inputs["q"], k_cache=inputs["k_cache"], v_cache=inputs["v_cache"], strides=inputs["strides"],
+        seq_len=inputs["seq_len"], prompt_len=inputs["prompt_len"], num_kv_heads=w.num_kv_heads,
+        max_seq_len=inputs["max_seq_len"], max_prompt_len=w.prompt_len, block_table=inputs["block_table"],
+        block_size=inputs["block_size"], num_blocks=inputs["block_table"].numel())
+    out, lse = dsa.alloc_outputs(prob)
+    n = w.n_att
+    cases = [
+        ("sliding_window", dsa.Diag(dsa.DSA_MASK_WINDOW, n)),
+        ("streaming_llm_4_sinks", dsa.Diag(dsa.DSA_MASK_WINDOW, n - 4, n_sink=4)),
+        ("diagonal_grid", dsa.Diag(dsa.DSA_MASK_GRID, w.window, n, w.grid_w, w.row_extra)),
+        ("diagonal_grid_4_sinks", dsa.Diag(dsa.DSA_MASK_GRID, w.window, n - 4, w.grid_w, w.row_extra, n_sink=4)),
+    ]
+    res = {"batch": w.batch, "n_att": n, "window": w.window}
+    row_bytes = w.num_kv_heads * w.head_dim * 2 * 2
+    for name, diag in cases:
+        ws = dsa.alloc_workspace(prob, diag)
+        _, cnt = dsa.dsa_debug_kept_indices(prob, diag, 0)
+        kept = int(cnt.sum().item())
+        secs, _ = time_calls(torch, lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws), 50, 5)
+        t = secs / 50
+        res[name] = {"us": round(t * 1e6, 2), "kept_rows_mean": round(kept / w.batch, 1),
+                     "GBs": round(kept * row_bytes / t / 1e9, 1), "frac_of_peak": round(kept * row_bytes / t / 1e9 / peak, 4)}
+    return res
+
+
 def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
                       modes=("dense", "sparse", "sparse_select", "dense_two_calls", "sparse_two_calls")):
     """Whole-image decode loop: 1024 image tokens after a 50-token prompt, `batch` requests (16: the
@@ -593,7 +625,7 @@ def run_ours(args):
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
-    per_config = decode_loop = decode_loop_large = selection = None
+    per_config = decode_loop = decode_loop_large = selection = masks = None
     if args.all_configs and rank == 0 and world == 1:
         del inputs, prob, out, lse
         torch.cuda.empty_cache()
@@ -603,6 +635,7 @@ def run_ours(args):
         decode_loop_large = decode_loop_bench(torch, dsa, synth, dev, batch=128,
                                               modes=("dense", "sparse", "sparse_select"))
         selection = selection_overhead(torch, dsa, synth, dev)
+        masks = mask_variants(torch, dsa, synth, dev, peak)
 
     if rank == 0:
         line = {
@@ -627,6 +660,7 @@ def run_ours(args):
             line["decode_loop"] = decode_loop
             line["decode_loop_batch128"] = decode_loop_large
             line["selection_overhead"] = selection
+            line["mask_variants"] = masks
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
