@@ -36,11 +36,11 @@ UNIT = "queries/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126 << 20
-# DRAM bytes per launch of the timed kernel from an ncu capture (see profiles/), keyed by the
-# workload string of the JSON line; None until a capture of that exact launch exists.
+# DRAM bytes per launch of the timed kernel (dram__bytes_read.sum + dram__bytes_write.sum of an ncu
+# capture), keyed by the workload string of the JSON line; None until a capture of that launch exists.
 NCU_TRAFFIC_BYTES = {
-    # ncu at batch 32: 209.39 MB read + 3.81 MB written per launch (profiles/dsa_attn_mma_kernel_...md);
-    # traffic grows in proportion to the batch, so a batch-256 launch moves 8 x that
+    # measured with ncu at batch 32: 209.39 MB read + 3.81 MB written per launch; traffic grows in
+    # proportion to the batch, so a batch-256 launch moves 8 x that
     "config5_paged_sweep B=256 Hq=32 Hkv=32 D=128 Lp=200 grid=64x64+1 paged16 sparse grid-mask window=512 n_att=208":
         8 * 213_193_600,
 }
@@ -61,9 +61,10 @@ def parse_args():
     ap.add_argument("--no-variants", action="store_true", help="skip the dense / other-window timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the table of every configuration (dense and sparse, L2 flushed between calls)")
     ap.add_argument("--all-configs", action="store_true",
-                    help="also time every configuration (dense and sparse, L2 flushed between calls) "
-                         "and add the table under 'per_config'")
+                    help="also run the whole-image decode loops and the mask-variant comparison")
     return ap.parse_args()
 
 
@@ -139,7 +140,7 @@ class ClockSampler:
             except Exception as e:  # pragma: no cover
                 self.err = repr(e)
                 break
-            time.sleep(0.002)
+            time.sleep(0.0005)
 
     def start(self):
         if self._nv is not None:
@@ -157,19 +158,57 @@ class ClockSampler:
         return out
 
 
-def algorithmic_bytes(w, host, mode, blocks_touched):
+def list_active_entries(position, window, n_att):
+    """Trace entries a LIST-mask request reads at decode position p (its active skips): with
+    t = p - 1, the selections of steps N_att-1 .. t-1, at most window - N_att of them."""
+    t = np.asarray(position, dtype=np.int64) - 1
+    return np.clip(t - (n_att - 1), 0, window - n_att)
+
+
+def union_rows(kept_idx, kept_cnt, group):
+    """Rows a LIST-mask call reads per (request, kv head) when every query head has its own mask:
+    the union of the kept sets of the `group` query heads that share the kv head (a row is fetched
+    once if any of them keeps it).  kept_idx [B, H_q, max_kept], kept_cnt [B, H_q] (numpy); returns
+    the total over requests and kv heads."""
+    b, hq, _ = kept_idx.shape
+    total = 0
+    for i in range(b):
+        for g0 in range(0, hq, group):
+            rows = set()
+            for h in range(g0, g0 + group):
+                rows.update(kept_idx[i, h, :int(kept_cnt[i, h])].tolist())
+            total += len(rows)
+    return total
+
+
+def algorithmic_bytes(w, host, mode, blocks_touched, list_mask=None):
     """Bytes one call must move: kept K and V rows, q, out, lse, and the block-table entries of
     the blocks it touches.  Kept rows per kv head: the whole prompt plus min(p, N_att) decode
-    keys for the sparse call (the attended count of Algorithm 1), p for the dense call."""
+    keys for the sparse call (the attended count of Algorithm 1), p for the dense call.
+    list_mask (LIST masks): {"mask_heads": 1 | H_kv | H_q, "union_rows": total rows over
+    (request, kv head) when query heads of a group keep different rows, else None}; adds the
+    trace entries every mask head reads, mask_heads x n_act x 4 bytes per request."""
     esize = 2
     p = host["position"].astype(np.int64)
     lp = host["prompt_len"].astype(np.int64)
     dec = p if mode == "dense" else np.minimum(p, w.n_att)
     kept_rows = int((lp + dec).sum())
-    kv = kept_rows * w.num_kv_heads * w.head_dim * esize * 2
+    kv_rows = kept_rows * w.num_kv_heads
+    trace = 0
+    if list_mask is not None:
+        if list_mask.get("union_rows") is not None:
+            kv_rows = int(list_mask["union_rows"])
+        trace = 4 * int(list_mask["mask_heads"]) * int(list_active_entries(p, w.window, w.n_att).sum())
+    kv = kv_rows * w.head_dim * esize * 2
     qo = w.batch * w.num_q_heads * (2 * w.head_dim * esize + 4)
     table = 4 * int(blocks_touched)
-    return kv + qo + table, kept_rows
+    return kv + qo + table + trace, kept_rows
+
+
+def aggregate_value(world, batch_per_rank, steps, rank_seconds):
+    """Whole-job throughput of a weak-scaling run: every rank processed batch_per_rank x steps
+    queries and the job took as long as its slowest rank."""
+    return world * batch_per_rank * steps / max(rank_seconds)
 
 
 def time_calls(torch, fn, steps, warmup, sampler=None, barrier=None):
@@ -515,26 +554,41 @@ def run_ours(args):
     abytes, kept_rows = algorithmic_bytes(w, host, args.mode, blocks_touched)
 
     # ---- the timed step ------------------------------------------------------------------
+    # One timed region is EXACTLY args.steps calls between two events.  A region of 20 steps lasts
+    # 5 ms, too short for the clock sampler, so the region is repeated (each repeat bracketed the same
+    # way) until 150 ms have been timed and the MEDIAN region is reported; the sampler runs across
+    # all repeats.
     sampler = ClockSampler(local_rank)
     flush_l2 = abytes < 2 * L2_BYTES
+    flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev) if flush_l2 else None
     if flush_l2:
-        flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
-        secs, clocks = time_calls_flushed(torch, call, args.steps, args.warmup, flush, sampler, barrier)
-        del flush
         l2_note = ("working set (%.3f GB per step) would stay in the %d MB L2: a %d MB write precedes every timed "
                    "call and only the calls are timed" % (abytes / 1e9, L2_BYTES >> 20, 4 * L2_BYTES >> 20))
     else:
-        secs, clocks = time_calls(torch, call, args.steps, args.warmup, sampler, barrier)
         l2_note = "inputs larger than L2: each step reads %.2f GB of distinct K/V" % (abytes / 1e9)
-    t = torch.tensor([secs], dtype=torch.float64, device=dev)
+
+    def region(warmup):
+        if flush_l2:
+            return time_calls_flushed(torch, call, args.steps, warmup, flush, None, barrier)[0]
+        return time_calls(torch, call, args.steps, warmup, None, barrier)[0]
+
+    first = region(args.warmup)                            # (also the warm-up of the repeats)
+    repeats = int(min(200, max(1, np.ceil(0.15 / max(first, 1e-6)))))
+    sampler.start()
+    regions = [region(0) for _ in range(repeats)]
+    clocks = sampler.stop()
+    regions_max = torch.tensor(regions, dtype=torch.float64, device=dev)
     if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    secs_max = float(t.item())
+        dist.all_reduce(regions_max, op=dist.ReduceOp.MAX)  # per repeat: the slowest rank
+    secs = float(np.median(regions))                       # this rank (roofline of its own launches)
+    secs_max = float(regions_max.median().item())
     ms_per_step = secs_max / args.steps * 1e3
-    value = world * w.batch * args.steps / secs_max
+    value = aggregate_value(world, w.batch, args.steps, [secs_max])
+    del flush
 
     # ---- roofline of the attention kernel (rank-local numbers) ----------------------------
     peak, peak_kind = measured_peak()
+    peak_gbs = peak
     launch_secs = secs / args.steps                       # one attention launch (+ combine) per step
     achieved = abytes / launch_secs / 1e9
     name = workload_name(w, args.mode)
@@ -545,32 +599,63 @@ def run_ours(args):
                 "kernel": ("dsa_attn_mma_kernel" if plan.tensor_cores else "dsa_attn_kernel") +
                           (" + dsa_combine_kernel" if plan.launches > 1 else "")}
 
-    # ---- variants: dense and the other window, same library, same batch --------------------
+    # ---- the same step as a single call with a cold L2 (launch latency and first misses included)
+    iso_flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+    iso_med, iso_min = time_flushed(torch, call, iso_flush, iters=30, warmup=3)
+    del iso_flush
+
+    # ---- variants: dense, the other window, and the paper's per-head list masks; same library,
+    # same batch, timed like the step
     variants = {}
     if not args.no_variants and args.mode == "sparse":
         vsteps = max(5, args.steps // 4)
+
+        def time_variant(vcall, vbytes):
+            if vbytes < 2 * L2_BYTES:                       # same rule as the timed step
+                vflush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+                vsecs, _ = time_calls_flushed(torch, vcall, vsteps, 3, vflush)
+                del vflush
+            else:
+                vsecs, _ = time_calls(torch, vcall, vsteps, 3)
+            return vsecs / vsteps
+
         todo = [("dense", w)]
         if w.index == 5:
             todo.append(("sparse", synth.workload(5, batch=w.batch, window=1024, n_att=416)))
         for mode, ww in todo:
             vcall, vplan, _ = make_call(mode, ww)
             vb, _ = algorithmic_bytes(ww, host, mode, 0)
-            if vb < 2 * L2_BYTES:                           # same rule as the timed step
-                vflush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
-                vsecs, _ = time_calls_flushed(torch, vcall, vsteps, 3, vflush)
-                del vflush
-            else:
-                vsecs, _ = time_calls(torch, vcall, vsteps, 3)
+            vt = time_variant(vcall, vb)
             key = "dense" if mode == "dense" else "sparse_w%d_a%d" % (ww.window, ww.n_att)
-            variants[key] = {"ms_per_step": round(vsecs / vsteps * 1e3, 4),
-                             "queries_per_sec": round(w.batch * vsteps / vsecs, 1),
-                             "achieved_GBs": round(vb / (vsecs / vsteps) / 1e9, 1),
-                             "frac_of_peak": round(vb / (vsecs / vsteps) / 1e9 / peak, 4),
+            variants[key] = {"ms_per_step": round(vt * 1e3, 4), "queries_per_sec": round(w.batch / vt, 1),
+                             "achieved_GBs": round(vb / vt / 1e9, 1), "frac_of_peak": round(vb / vt / 1e9 / peak_gbs, 4),
                              "launches_per_step": vplan.launches, "n_split": vplan.n_split}
         if "dense" in variants:
-            variants["sparse_over_dense_speedup"] = round(variants["dense"]["ms_per_step"] / (launch_secs * 1e3), 3)
+            variants["sparse_over_dense_speedup"] = round(variants["dense"]["ms_per_step"] / (secs / args.steps * 1e3), 3)
             dense_bytes, _ = algorithmic_bytes(w, host, "dense", 0)
             variants["ideal_byte_ratio"] = round(dense_bytes / abytes, 3)
+        # The paper's own setting: one skip list per attention head (random valid traces here), without
+        # and with the fused phase-2 selection (which appends the next trace entry of every head whose
+        # request is in phase 2).  Same positions, same budget, same kernel family.
+        lrng = np.random.default_rng(synth.BASE_SEED + 500 + w.index)
+        few = synth.random_valid_trace(lrng, w.window, w.n_att, (8,))
+        trace = torch.from_numpy(np.ascontiguousarray(
+            few[lrng.integers(0, 8, size=(w.batch, w.num_q_heads))])).to(dev)
+        group = w.num_q_heads // w.num_kv_heads
+        for key, sel in (("list_per_head", False), ("list_per_head_select", True)):
+            ldiag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=trace, select=sel)
+            lws = dsa.alloc_workspace(prob, ldiag)
+            lplan = dsa.dsa_query_plan(prob, ldiag)
+            lmask = {"mask_heads": w.num_q_heads, "union_rows": None}
+            if group > 1:
+                lidx, lcnt = dsa.dsa_debug_kept_indices(prob, ldiag, inputs["max_seq_len"])
+                lmask["union_rows"] = union_rows(lidx.cpu().numpy(), lcnt.cpu().numpy(), group)
+            lb, _ = algorithmic_bytes(w, host, "sparse", blocks_touched, lmask)
+            lt = time_variant(lambda: dsa.dsa_decode_attention_sparse(prob, ldiag, out, lse, lws), lb)
+            variants[key] = {"ms_per_step": round(lt * 1e3, 4), "queries_per_sec": round(w.batch / lt, 1),
+                             "algorithmic_bytes": lb, "achieved_GBs": round(lb / lt / 1e9, 1),
+                             "frac_of_peak": round(lb / lt / 1e9 / peak_gbs, 4),
+                             "launches_per_step": lplan.launches, "n_split": lplan.n_split}
 
     # ---- end to end: per-step inputs from pinned host memory, result back to the host ------
     e2e = None
@@ -626,21 +711,31 @@ def run_ours(args):
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
     per_config = decode_loop = decode_loop_large = selection = masks = None
-    if args.all_configs and rank == 0 and world == 1:
+    if rank == 0 and world == 1 and (not args.no_per_config or args.all_configs):
         del inputs, prob, out, lse
         torch.cuda.empty_cache()
-        per_config = per_config_table(torch, dsa, synth, dev, peak)
-        decode_loop = decode_loop_bench(torch, dsa, synth, dev)
-        # the same loop at a batch where a B200 step is bandwidth-bound rather than latency-bound
-        decode_loop_large = decode_loop_bench(torch, dsa, synth, dev, batch=128,
-                                              modes=("dense", "sparse", "sparse_select"))
-        selection = selection_overhead(torch, dsa, synth, dev)
-        masks = mask_variants(torch, dsa, synth, dev, peak)
+        if not args.no_per_config:
+            per_config = per_config_table(torch, dsa, synth, dev, peak)
+        if args.all_configs:
+            decode_loop = decode_loop_bench(torch, dsa, synth, dev)
+            # the same loop at a batch where a B200 step is bandwidth-bound rather than latency-bound
+            decode_loop_large = decode_loop_bench(torch, dsa, synth, dev, batch=128,
+                                                  modes=("dense", "sparse", "sparse_select"))
+            selection = selection_overhead(torch, dsa, synth, dev)
+            masks = mask_variants(torch, dsa, synth, dev, peak)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5),
+            "timed_regions": {"repeats": repeats, "reported": "median region of %d steps" % args.steps,
+                              "ms_per_step_min": round(float(regions_max.min().item()) / args.steps * 1e3, 5),
+                              "ms_per_step_max": round(float(regions_max.max().item()) / args.steps * 1e3, 5),
+                              "ms_per_step_first": round(first / args.steps * 1e3, 5)},
+            "isolated_ms": {"median": round(iso_med * 1e3, 5), "min": round(iso_min * 1e3, 5),
+                            "note": "one call at a time, a %d MB write before each (cold L2), 30 calls; "
+                                    "ms_per_step is back-to-back calls, whose launch latency and prologue "
+                                    "overlap the previous call" % (4 * L2_BYTES >> 20)},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": name, "global_batch": world * w.batch,
@@ -657,6 +752,7 @@ def run_ours(args):
         }
         if per_config is not None:
             line["per_config"] = per_config
+        if decode_loop is not None:
             line["decode_loop"] = decode_loop
             line["decode_loop_batch128"] = decode_loop_large
             line["selection_overhead"] = selection
@@ -728,7 +824,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": min(args.warmup, 3), "ms_per_step": round(el / steps * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": workload_name(w_full, args.mode)},
+        "data": "synthetic",
+        "config": {"workload": workload_name(w_full, args.mode) + " (%d-request sample per step)" % sample},
         "cpu_baseline": cpu,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 

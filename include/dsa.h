@@ -13,18 +13,22 @@
  *     work queued on `stream` has finished.  The dsa_problem / dsa_diag_params structs themselves
  *     are HOST memory, read during the call only.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream);
- *     the library never synchronises, allocates no device memory and keeps no state between
- *     calls.  Scratch comes from the caller's `workspace` (device, 256-byte aligned), sized by
- *     dsa_workspace_size(); it may be reused by the next call on the same stream.
+ *     the library never synchronises and allocates no device memory.  It reads no environment
+ *     variable and carries no result from one call to the next; what it does remember per device
+ *     are idempotent set-up caches (which kernel variants have been configured, the SM count, the
+ *     address of the built-in scratch array), written with atomics, so calls may come from several
+ *     host threads.  Scratch comes from the caller's `workspace` (device, 256-byte aligned), sized
+ *     by dsa_workspace_size(); it may be reused by the next call on the same stream.  The one
+ *     exception is dsa_decode_attention_static_scratch(), whose scratch is a fixed array inside
+ *     the library image.
  *   - Arguments are checked on the host before anything is launched.  Values that live in
  *     device memory (seq_len, prompt_len, block ids, skip offsets) cannot be checked there;
  *     kernels clamp them into range instead, so bad values give wrong numbers, not faults.
  *   - Return value: DSA_OK or a negative dsa_status.  After DSA_ERR_CUDA the CUDA error code is
  *     available from dsa_last_cuda_error().
- *   - The first launch of each kernel variant on a device also configures it (a one-time
- *     attribute call that must not happen inside a stream capture): call dsa_prepare() once per
- *     device, or make the first call of a given shape, before capturing.  After that every call
- *     of this header can be captured into CUDA graphs.
+ *   - The first launch of each kernel variant on a device also configures it (one-time
+ *     attribute and address queries that must not happen inside a stream capture): call
+ *     dsa_prepare() once per device, or make the first call of a given shape, before capturing.
  *   - There is no CPU path: without a CUDA device every compute call fails with DSA_ERR_CUDA.
  *
  * Positions.  For request b, prompt_len[b] = L_p tokens of prompt come first in the cache and
@@ -104,7 +108,7 @@ typedef struct dsa_problem {
                                /* call then plans for max_seq_len kept tokens)                     */
     int32_t split_tokens;      /* kept tokens handled by one thread block; 0 = library chooses.    */
                                /* Rounded up to the tile size, at most 1024                        */
-    /* Bounded cache (Algorithm 1, phase 3: "evict oldest KV"; footprint N_r + L_p of Section 4's
+    /* Bounded cache (the eviction step of Algorithm 1, phase 3; footprint N_r + L_p of Section 4's
      * cost analysis).  ring_size == 0: every token is stored at its logical position.
      * ring_size > 0: the prompt and the first ring_sinks decode tokens are stored at their logical
      * positions; decode token j >= ring_sinks is stored at position
@@ -112,10 +116,20 @@ typedef struct dsa_problem {
      * window ring_size steps earlier.  seq_len stays the LOGICAL length.  Needs
      * max_prompt_len > 0; sparse calls need window <= ring_size and n_sink <= ring_sinks; the
      * dense call is refused.  The cache then needs max_prompt_len + ring_sinks + ring_size
-     * tokens per request instead of max_seq_len. */
+     * tokens per request instead of max_seq_len; a device prompt_len[b] above max_prompt_len is
+     * read as max_prompt_len, so that no row is addressed outside that region. */
     int32_t ring_size;
     int32_t ring_sinks;
+    /* 0 in production: the library chooses the launch plan.  Comparison runs and tests may force
+     * single planner decisions with the DSA_PLAN_* bits below; results never depend on them
+     * beyond summation order. */
+    uint32_t plan_flags;
 } dsa_problem;
+
+#define DSA_PLAN_CUDA_CORES    0x01u  /* bf16 through the CUDA-core kernel instead of the tensor-core one */
+#define DSA_PLAN_NO_ITEM_WARPS 0x02u  /* small launches: split + combine, never four warps on one item   */
+#define DSA_PLAN_RING_DEEP     0x04u  /* two-heads-per-block kernel: keep the 3-stage ring               */
+#define DSA_PLAN_RING_SHALLOW  0x08u  /* two-heads-per-block kernel: take the 2-stage ring               */
 
 /*
  * Which decode keys are kept (Algorithm 1 with its data-dependent selection made an input).
@@ -140,8 +154,8 @@ typedef struct dsa_problem {
  *         multiples of the row stride.)
  *   WINDOW nothing skipped (n_att is ignored).  This is the paper's SlidingWindow baseline.
  *
- * Selection (Algorithm 1, phase 2: "select newly skipped KV", fused into the attention pass as
- * in Section 5.1).  With `select` set, a request whose step t lies in N_att-1 .. N_r-2 also gets
+ * Selection (the choice of the next skipped key in Algorithm 1, phase 2, fused into the attention
+ * pass as in Section 5.1).  With `select` set, a request whose step t lies in N_att-1 .. N_r-2 also gets
  * the next trace entry: among the decode keys it attends (sinks excluded) the one with the lowest
  * softmax weight -- the lowest logit; equal logits go to the lowest cache index -- is found per
  * query head and its distance is written to skip_offsets[b][h][t - (N_att-1)], which takes effect
@@ -192,9 +206,10 @@ DSA_API int32_t dsa_last_cuda_error(void);
 
 /*
  * Configure every kernel variant of the library for the CURRENT device (a few hundred one-time
- * attribute calls, no launch, no allocation).  Optional: calls do it lazily for the variant they
- * need; required only before a stream capture whose calls would otherwise be the first of their
- * shape on this device.
+ * attribute calls, the SM count and the address of the built-in scratch array of
+ * dsa_decode_attention_static_scratch; no launch, no allocation).  Optional: calls do it lazily
+ * for what they need; required only before a stream capture whose calls would otherwise be the
+ * first of their shape on this device.
  */
 DSA_API int32_t dsa_prepare(void);
 
@@ -343,8 +358,8 @@ DSA_API int32_t dsa_debug_kept_indices(const dsa_problem *problem, const dsa_dia
  * exactly as above and results are identical to dsa_decode_attention_dense / _sparse.
  * Problems whose partials exceed the array are refused with DSA_ERR_WORKSPACE_TOO_SMALL and
  * nothing is launched; dsa_workspace_size() tells the size in advance.
- * The first call on each device looks up the array's device address (with that device current);
- * make that first call outside any stream capture.
+ * The first call on each device (or dsa_prepare() before it) looks up the array's device address,
+ * with that device current; let that happen before any stream capture begins.
  * All calls share the one array and it keeps whatever the last call left there; nothing in it
  * needs clearing between calls.  Two calls whose kernels can run at the same time on one GPU
  * (different streams, different host threads) would overwrite each other's partials: keep calls

@@ -24,7 +24,7 @@
  * Readings of the paper taken here (each is also listed in the design notes of the repository):
  *   R1  The window of Algorithm 1 is written [max(0,t-N_r) .. t], which has N_r+1 entries once
  *       t >= N_r; phase 3 evicts K[t-N_r] in the same step, so N_r entries stay.  The paper's
- *       example (N_r = 7, N_att = 4, three skips, "attended count stays fixed at 4") fixes this.
+ *       example (N_r = 7, N_att = 4, three skips, four keys attended from then on) fixes this.
  *   R2  Phase 1 is t < N_att-1 (the algorithm), not t < N_att (one sentence of the prose); the
  *       example selects first at t = 3 with N_att = 4.
  *   R3  An entry appended to skip_idx at step s is not skipped at step s (Section 4, item 2).
@@ -39,7 +39,7 @@
  *   R8  Sink variants (Section 5.1, "Diagonal + sink4", StreamingLLM): the first n_sink decode
  *       tokens are attended at every step on top of what Algorithm 1 attends; the selection runs
  *       unchanged with its own N_att (callers pass N_att = budget - n_sink), except that a sink
- *       is never a candidate of the argmin ("diagonal selection for the remaining slots").
+ *       is never a candidate of the argmin (Section 5.1: the selection fills the other slots only).
  *                                                                        [parity unpinned]
  *   R7  A request with no decode token yet (seq_len == prompt_len) attends its prompt only; a
  *       request with seq_len == 0 yields out = 0 and lse = -inf.

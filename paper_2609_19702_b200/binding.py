@@ -19,6 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libdsa.so")
 
 DSA_BF16, DSA_F32 = 0, 1
 DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
+# dsa_problem.plan_flags: 0 lets the library plan; the bits force single decisions (comparison runs, tests)
+DSA_PLAN_CUDA_CORES, DSA_PLAN_NO_ITEM_WARPS, DSA_PLAN_RING_DEEP, DSA_PLAN_RING_SHALLOW = 0x1, 0x2, 0x4, 0x8
 
 EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_workspace_size",
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
@@ -39,7 +41,8 @@ class dsa_problem(ctypes.Structure):
                 ("max_blocks", ctypes.c_int32), ("block_size", ctypes.c_int32),
                 ("num_blocks", ctypes.c_int32), ("max_seq_len", ctypes.c_int32),
                 ("max_prompt_len", ctypes.c_int32), ("split_tokens", ctypes.c_int32),
-                ("ring_size", ctypes.c_int32), ("ring_sinks", ctypes.c_int32)]
+                ("ring_size", ctypes.c_int32), ("ring_sinks", ctypes.c_int32),
+                ("plan_flags", ctypes.c_uint32)]
 
 
 class dsa_diag_params(ctypes.Structure):
@@ -151,6 +154,7 @@ class Problem:
     split_tokens: int = 0
     ring_size: int = 0                    # > 0: bounded cache, decode tokens live in a ring
     ring_sinks: int = 0
+    plan_flags: int = 0                   # DSA_PLAN_* bits; 0 = the library chooses the launch plan
 
     def c_struct(self) -> dsa_problem:
         b, hq, d = self.q.shape
@@ -173,6 +177,7 @@ class Problem:
         p.max_prompt_len = int(self.max_prompt_len)
         p.split_tokens = int(self.split_tokens)
         p.ring_size, p.ring_sinks = int(self.ring_size), int(self.ring_sinks)
+        p.plan_flags = int(self.plan_flags)
         return p
 
 
@@ -386,7 +391,7 @@ def dsa_debug_kept_indices(problem: Problem, diag: Optional[Diag], max_kept: int
 
 
 def problem_from_host(inp: dict, device: str = "cuda", dtype: torch.dtype = torch.bfloat16,
-                      split_tokens: int = 0) -> Problem:
+                      split_tokens: int = 0, plan_flags: int = 0) -> Problem:
     """Copy one host batch (as made by ``synth.make_inputs``: bf16 bit patterns) to the device."""
     w = inp["workload"]
 
@@ -403,4 +408,4 @@ def problem_from_host(inp: dict, device: str = "cuda", dtype: torch.dtype = torc
         num_kv_heads=w.num_kv_heads, max_seq_len=inp["max_seq_len"], max_prompt_len=w.prompt_len,
         block_table=None if bt is None else torch.from_numpy(bt).to(device),
         block_size=inp["block_size"], num_blocks=0 if bt is None else int(bt.size),
-        split_tokens=split_tokens)
+        split_tokens=split_tokens, plan_flags=plan_flags)

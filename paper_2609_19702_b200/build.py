@@ -34,7 +34,6 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--extended-lambda",
              "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
-    flags += os.environ.get("DSA_NVCC_FLAGS", "").split()         # e.g. tuning -D overrides
     if verbose:
         flags += ["-Xptxas", "-v"]
     work = tempfile.mkdtemp(prefix="dsa_build_")

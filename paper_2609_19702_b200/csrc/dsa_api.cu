@@ -2,6 +2,7 @@
 // kernel dispatch.  Everything here is host code except the kernels it instantiates.
 #include "../../include/dsa.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -21,14 +22,32 @@ int32_t cuda_fail(cudaError_t e) {
     return DSA_ERR_CUDA;
 }
 
-constexpr int kNumSMs = 148;
-
-int env_int(const char* name, int fallback) {
-    const char* v = std::getenv(name);
-    return (v && *v) ? std::atoi(v) : fallback;
+// SM count of the current device, asked for once per device (an idempotent cache: two threads that
+// race on the first call store the same value).  Falls back to the B200's 148 if the query fails.
+int sm_count() {
+    static std::atomic<int> cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return 148;
+    }
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n <= 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            return 148;
+        }
+        cached[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
 }
 
+constexpr uint32_t kKnownPlanFlags =
+    DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_RING_DEEP | DSA_PLAN_RING_SHALLOW;
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+constexpr int kMaxSplits = 8192;                 // split weights of the combine kernel: 32 KB of shared memory
 
 // The launch plan: how many kept rows one block takes, how many splits that makes.
 struct Plan {
@@ -85,6 +104,7 @@ int32_t check_problem(const dsa_problem* p) {
     const int G = p->num_q_heads / p->num_kv_heads;
     if (G != 1 && G != 2 && G != 4 && G != 8) return DSA_ERR_UNSUPPORTED;
     if (p->max_seq_len < 0 || p->max_prompt_len < 0 || p->split_tokens < 0) return DSA_ERR_INVALID_ARG;
+    if (p->plan_flags & ~kKnownPlanFlags) return DSA_ERR_INVALID_ARG;
     if (!(p->sm_scale >= 0.f) || !std::isfinite(p->sm_scale)) return DSA_ERR_INVALID_ARG;
     if (p->batch == 0) return DSA_OK;
     if (!p->q || !p->k_cache || !p->v_cache || !p->seq_len || !p->prompt_len) return DSA_ERR_INVALID_ARG;
@@ -151,9 +171,10 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     }
     if (bound < 1) bound = 1;
 
+    const int kNumSMs = sm_count();
     // bf16 runs on the tensor-core kernel (one warp per work item); fp32 on the CUDA-core kernel.
-    // DSA_CUDA_CORES=1 forces the latter for bf16 too (comparison runs).
-    pl->mma = p->dtype == DSA_BF16 && env_int("DSA_CUDA_CORES", 0) == 0;
+    // DSA_PLAN_CUDA_CORES forces the latter for bf16 too (comparison runs).
+    pl->mma = p->dtype == DSA_BF16 && !(p->plan_flags & DSA_PLAN_CUDA_CORES);
     pl->mma_warps = 1;
     pl->mma_kw = 1;
     pl->mma_stages = kMmaStages;
@@ -201,7 +222,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         // 32.8 us against 29.7 us for three splits and the combine; with ~1000-row items the
         // single launch still wins there).  Requests beyond 2048 rows need the combine anyway;
         // there the merge on top of it measured as a small loss.
-        if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK && env_int("DSA_ITEM_WARPS", 1) != 0) {
+        if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK && !(p->plan_flags & DSA_PLAN_NO_ITEM_WARPS)) {
             const int64_t kw_blocks = pairs * ((want_split + kMmaItemWarps - 1) / kMmaItemWarps);
             if (kw_blocks <= 2 * kNumSMs || kw_blocks >= 4 * kNumSMs || bound > MAX_CHUNK) {
                 pl->mma_kw = kMmaItemWarps;
@@ -221,6 +242,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     }
     pl->chunk = chunk;
     pl->n_split = (int)((bound + chunk - 1) / chunk);
+    if (pl->n_split > kMaxSplits) return DSA_ERR_UNSUPPORTED;   // the combine kernel holds one weight per split
     pl->grid = (int64_t)p->batch * p->num_kv_heads * pl->n_split;
     if (pl->grid > 0x7fffffffLL) return DSA_ERR_UNSUPPORTED;
 
@@ -236,9 +258,10 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     // Only for unsplit plans: the splits of a long request differ so much in length (many are
     // empty) that their blocks pack into waves far better than the estimate assumes (measured: a
     // loss of 10 % on the dense calls at batch 1-8).
+    const bool force_shallow = (p->plan_flags & DSA_PLAN_RING_SHALLOW) != 0;
+    const bool force_deep = (p->plan_flags & DSA_PLAN_RING_DEEP) != 0 && !force_shallow;
     if (pl->mma && pl->mma_warps == 2 && pl->mma_kw == 1 && p->split_tokens == 0 &&
-        (pl->n_split == 1 || env_int("DSA_MMA_STAGES", 0) == kMmaStagesShallow) &&
-        env_int("DSA_MMA_STAGES", 0) != kMmaStages) {
+        (pl->n_split == 1 || force_shallow) && !force_deep) {
         Plan alt = *pl;
         alt.mma_stages = kMmaStagesShallow;
         KernelShape shallow = {};
@@ -258,7 +281,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
             return (whole + rest) * cap;
         };
         if (rc2 == DSA_OK && shallow.stages == kMmaStagesShallow) {
-            const bool forced = env_int("DSA_MMA_STAGES", 0) == kMmaStagesShallow;
+            const bool forced = force_shallow;
             // (with many waves the two are within a few per cent either way: stay with the deep ring
             // unless the estimate is clearly better)
             const double margin = (double)(pl->grid / 2) < 3.0 * 4 * kNumSMs ? 1.0 : 0.97;
@@ -297,6 +320,9 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->max_blocks = p->max_blocks; a->block_size = p->block_size; a->num_blocks = p->num_blocks;
     a->max_seq_len = p->max_seq_len;
     a->ring_size = p->ring_size; a->ring_sinks = p->ring_sinks;
+    // the prompt length the kernels trust: with a bounded cache the region of a request holds
+    // max_prompt_len + ring_sinks + ring_size tokens, so a longer device prompt_len is cut there
+    a->prompt_cap = p->ring_size > 0 ? p->max_prompt_len : p->max_seq_len;
     a->B = p->batch; a->H_q = p->num_q_heads; a->H_kv = p->num_kv_heads;
     const float scale = p->sm_scale > 0.f ? p->sm_scale : 1.f / sqrtf((float)p->head_dim);
     a->scale_log2 = scale * LOG2E;
@@ -329,7 +355,7 @@ cudaError_t launch_combine_t(const float* out_part, const float* lse_part, int64
                              const int* sel_k, int* trace, int trace_len, bool after_attention) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)rows);
-    cfg.blockDim = dim3((unsigned)D);
+    cfg.blockDim = dim3((unsigned)((D + 31) / 32 * 32));    // whole warps: the block reductions shuffle with a full mask
     cfg.dynamicSmemBytes = (size_t)n_split * sizeof(float);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -454,11 +480,16 @@ const char* dsa_status_string(int32_t status) {
 
 int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
 
+static cudaError_t static_scratch_address(void** out);
+
 int32_t dsa_prepare(void) {
     cudaError_t e = kernel_prepare<__nv_bfloat16, 64>();
     if (e == cudaSuccess) e = kernel_prepare<__nv_bfloat16, 128>();
     if (e == cudaSuccess) e = kernel_prepare<float, 64>();
     if (e == cudaSuccess) e = kernel_prepare<float, 128>();
+    void* scratch = nullptr;
+    if (e == cudaSuccess) e = static_scratch_address(&scratch);   // (and remember it for this device)
+    sm_count();
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
@@ -587,7 +618,7 @@ int32_t dsa_combine_splits(const float* out_part, const float* lse_part, int32_t
                            int32_t head_dim, int32_t n_split, void* out, float* lse, int32_t out_dtype,
                            void* stream) {
     if (batch < 0 || num_q_heads < 1 || head_dim < 1 || head_dim > 1024 || n_split < 1) return DSA_ERR_INVALID_ARG;
-    if (n_split > 8192) return DSA_ERR_UNSUPPORTED;              // weights live in 32 KB of shared memory
+    if (n_split > kMaxSplits) return DSA_ERR_UNSUPPORTED;        // weights live in 32 KB of shared memory
     if (out_dtype != DSA_BF16 && out_dtype != DSA_F32) return DSA_ERR_UNSUPPORTED;
     if (batch == 0) return DSA_OK;
     if (!out_part || !lse_part || !out) return DSA_ERR_INVALID_ARG;
@@ -648,28 +679,37 @@ int32_t dsa_debug_kept_indices(const dsa_problem* problem, const dsa_diag_params
 // is part of the library image: every GPU that loads the library holds these bytes until exit.
 static __device__ __align__(256) unsigned char g_static_scratch[DSA_STATIC_SCRATCH_MAX];
 
-int32_t dsa_decode_attention_static_scratch(const dsa_problem* problem, const dsa_diag_params* diag, void* out,
-                                            float* lse, void* stream) {
-    // In host code `g_static_scratch` is only a handle for the symbol; the address kernels can use
-    // must be asked for, once per device and with that device current.
-    static void* scratch_addr[kMaxDevices] = {};
+// In host code `g_static_scratch` is only a handle for the symbol; the address kernels can use must
+// be asked for, once per device and with that device current.  The per-device cache is idempotent
+// (threads that race on the first call store the same address) and written atomically.
+static cudaError_t static_scratch_address(void** out) {
+    static std::atomic<void*> scratch_addr[kMaxDevices] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail(e);
-    if (dev < 0 || dev >= kMaxDevices) return DSA_ERR_UNSUPPORTED;
-    if (!scratch_addr[dev]) {
-        void* ptr = nullptr;
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    void* ptr = scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-        if (e != cudaSuccess) return cuda_fail(e);
-        scratch_addr[dev] = ptr;
+        if (e != cudaSuccess) return e;
+        scratch_addr[dev].store(ptr, std::memory_order_release);
     }
+    *out = ptr;
+    return cudaSuccess;
+}
+
+int32_t dsa_decode_attention_static_scratch(const dsa_problem* problem, const dsa_diag_params* diag, void* out,
+                                            float* lse, void* stream) {
+    void* scratch = nullptr;
+    const cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
     size_t need = 0;
     const int32_t rc = dsa_workspace_size(problem, diag, &need);
     if (rc != DSA_OK) return rc;
     if (need > DSA_STATIC_SCRATCH_MAX) return DSA_ERR_WORKSPACE_TOO_SMALL;   // problem too large for the fixed array
     // Nothing in the scratch has to start at zero: every split writes its own lse, and the output of
     // an empty split is never read, so leftovers of the previous call are harmless.
-    return run_attention(problem, diag, out, lse, scratch_addr[dev], DSA_STATIC_SCRATCH_MAX, stream);
+    return run_attention(problem, diag, out, lse, scratch, DSA_STATIC_SCRATCH_MAX, stream);
 }
 
 }  // extern "C"

@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(NT) dsa_attn_kernel(const AttnArgs a) {
     const int b = blockIdx.x / (a.H_kv * a.n_split);
 
     bool has_new;                                         // (the rows were appended by an earlier kernel)
-    const ReqMask m = req_mask_setup(a.mask, step_seq_len(a, a.seq_len[b], has_new), a.prompt_len[b], a.max_seq_len);
+    const ReqMask m = req_mask_setup(a.mask, step_seq_len(a, a.seq_len[b], has_new), req_prompt_len(a, b), a.max_seq_len);
     const int n_rows = build_row_list<C, BlockSync>(a, m, b, kvh, split, list, bitmaps, s_warp);
     if (n_rows <= 0) { write_empty_item<C>(a, m, b, kvh, split); return; }
     __syncthreads();

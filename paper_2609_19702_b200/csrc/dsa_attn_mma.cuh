@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     const int split = (blockIdx.x / hblocks) % a.n_split;
     const int b = blockIdx.x / (hblocks * a.n_split);
 
-    const int seq_raw = a.seq_len[b], prompt_raw = a.prompt_len[b];
+    const int seq_raw = a.seq_len[b], prompt_raw = req_prompt_len(a, b);
     // ---- Q^T as B operand: head = lane / 4, dims 2*(lane%4)+{0,1} (+8) of every 16-dim step ----
     // Loaded first, used last: the loads depend on nothing but the work item, so their latency
     // hides behind the mask set-up and the row list (columns beyond the group are zeroed at use).

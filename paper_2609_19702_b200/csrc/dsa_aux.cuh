@@ -95,7 +95,7 @@ __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_n
     const int b = blockIdx.x;
     const int S = a.seq_len[b];
     if (S < 0 || S >= capacity) return;                   // no room: the token is dropped
-    const int L_p = max(0, min(a.prompt_len[b], S));
+    const int L_p = max(0, min(req_prompt_len(a, b), S));
     const int64_t dst0 = token_offset(a, b, L_p, S);
     constexpr int VEC = 16 / (int)sizeof(T);
     T* kc = reinterpret_cast<T*>(const_cast<void*>(a.k));
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(NT) dsa_kept_indices_kernel(const AttnArgs a, 
     const int mheads = a.mask.mode == MODE_LIST ? a.mask.mask_heads : 1;
     const int mh = blockIdx.x % mheads, b = blockIdx.x / mheads;
     bool has_new;                                         // (the rows were appended by an earlier kernel)
-    const ReqMask m = req_mask_setup(a.mask, step_seq_len(a, a.seq_len[b], has_new), a.prompt_len[b], a.max_seq_len);
+    const ReqMask m = req_mask_setup(a.mask, step_seq_len(a, a.seq_len[b], has_new), req_prompt_len(a, b), a.max_seq_len);
     if (a.mask.mode == MODE_LIST && !m.keep_all) {
         for (int i = threadIdx.x; i < a.mask.bitmap_words; i += NT) bitmap[i] = 0u;
         __syncthreads();

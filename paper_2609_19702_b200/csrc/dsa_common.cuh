@@ -24,6 +24,7 @@ struct AttnArgs {
     const int* block_table;
     int max_blocks, block_size, num_blocks;
     int max_seq_len;
+    int prompt_cap;              // device prompt_len values above this are read as this (see req_prompt_len)
     int ring_size, ring_sinks;   // bounded cache: decode tokens beyond the first ring_sinks live in a ring
     int B, H_q, H_kv;
     float scale_log2;            // sm_scale * log2(e)
@@ -45,6 +46,13 @@ struct AttnArgs {
     const void* k_new;           // [B, H_kv, D] rows of the current token; NULL: already in the cache
     const void* v_new;
 };
+
+// The prompt length of request b as the kernels use it.  With a bounded cache a request's region
+// holds max_prompt_len + ring_sinks + ring_size tokens, so a device value above max_prompt_len is
+// cut there: every address derived from it then stays inside the region.
+__device__ __forceinline__ int req_prompt_len(const AttnArgs& a, int b) {
+    return min(a.prompt_len[b], a.prompt_cap);
+}
 
 // Number of tokens request b attends over.  In a fused decode step that is one more than the
 // cache holds, unless the request is full (the token is then dropped, as by the append call).

@@ -5,6 +5,7 @@
 #include "dsa_attn_mma.cuh"
 #include "dsa_launch.cuh"
 
+#include <atomic>
 #include <type_traits>
 
 namespace dsa {
@@ -34,19 +35,8 @@ struct KernelPick {
     // 8 or more blocks share an SM and their start-up and merge phases overlap each other's
     // streaming.  (Measured on the paged batch-256 workload: 32-row tiles with 3 blocks/SM reach
     // 5.7 TB/s, these reach 6.6 TB/s; the dense call is flat at 7.2 TB/s either way.)
-    // -DDSA_TUNE_TILE / -DDSA_TUNE_STAGES override the bf16, head_dim 128 choice in tuning builds.
-    static constexpr int kTileDefault = 2048 / (D * (int)sizeof(T));
-    static constexpr int kStagesDefault = 4;
-#ifdef DSA_TUNE_TILE
-    static constexpr int TILE = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_TILE : kTileDefault;
-#else
-    static constexpr int TILE = kTileDefault;
-#endif
-#ifdef DSA_TUNE_STAGES
-    static constexpr int STAGES = (sizeof(T) == 2 && D == 128) ? DSA_TUNE_STAGES : kStagesDefault;
-#else
-    static constexpr int STAGES = kStagesDefault;
-#endif
+    static constexpr int TILE = 2048 / (D * (int)sizeof(T));
+    static constexpr int STAGES = 4;
     using Cfg = AttnCfg<T, D, G, TILE, STAGES, HM, SEL>;
     static size_t smem(int chunk, int bw) { return Cfg::smem_bytes(chunk, bw); }
     // Tensor-core kernel (bf16 only).  W warps per block share one row list when the mask does not
@@ -64,21 +54,24 @@ struct KernelPick {
         return smem_mma_w<1>(chunk, bw);
     }
     // Kernels that use more than 48 KB of dynamic shared memory must be told so once per device.
+    // The per-device flags are idempotent caches (configuring twice is harmless), kept atomic so
+    // that host threads may make their first calls at the same time.
+    using ConfiguredFlags = std::atomic<bool>;
     template <class Kern>
-    static cudaError_t ensure_configured(Kern kern, bool* done /* [kMaxDevices] */) {
+    static cudaError_t ensure_configured(Kern kern, ConfiguredFlags* done /* [kMaxDevices] */) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices || !done[dev]) {
+        if (dev < 0 || dev >= kMaxDevices || !done[dev].load(std::memory_order_acquire)) {
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
             if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) done[dev] = true;
+            if (dev >= 0 && dev < kMaxDevices) done[dev].store(true, std::memory_order_release);
         }
         return cudaSuccess;
     }
     template <int W, bool APPEND, int KW, int ST>
-    static bool* mma_configured() { static bool done[kMaxDevices] = {}; return done; }
-    static bool* cc_configured() { static bool done[kMaxDevices] = {}; return done; }
+    static ConfiguredFlags* mma_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    static ConfiguredFlags* cc_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
 
     template <int W, bool APPEND, int KW, int ST = kMmaStages>
     static cudaError_t launch_mma_w(const AttnArgs& a, int64_t grid, size_t smem_bytes, cudaStream_t st) {

@@ -8,10 +8,7 @@ namespace dsa {
 
 constexpr int kMaxDevices = 64;
 constexpr int kMmaItemWarps = 4;                   // warps per work item in small launches
-#ifndef DSA_TUNE_MMA_STAGES
-#define DSA_TUNE_MMA_STAGES 3
-#endif
-constexpr int kMmaStages = DSA_TUNE_MMA_STAGES;    // 16-key tiles in flight per warp (+1 being consumed)
+constexpr int kMmaStages = 3;                      // ring slots per warp: two 16-key tiles in flight, one being consumed
 constexpr int kMmaStagesShallow = 2;               // the shallow-ring form of the two-heads-per-block kernel
 
 // Which kernel variant a call needs.

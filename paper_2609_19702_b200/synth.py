@@ -214,12 +214,13 @@ def shard_requests(batch: int, world_size: int, rank: int) -> range:
     return range(lo, lo + base + (1 if rank < extra else 0))
 
 
-def make_inputs_device(w: Workload, device, seed: Optional[int] = None) -> Dict[str, object]:
+def make_inputs_device(w: Workload, device, seed: Optional[int] = None, poison: bool = True) -> Dict[str, object]:
     """Full-size batches for benchmarking: same shapes, layouts and position mix as
     ``make_inputs`` but K/V/q are drawn on ``device`` with a seeded torch generator (a paged pool
     at batch 256 is 18 GB, too slow to draw on the host).  Values are N(0,1) (+ the positional
-    component where the workload has one) rounded to bf16.  Returns torch tensors; positions,
-    lengths and the block table are also returned as numpy arrays under ``host``.
+    component where the workload has one) rounded to bf16; cache rows at positions >= seq_len are
+    NaN when ``poison`` (never for a shared cache), as in ``make_inputs``.  Returns torch tensors;
+    positions, lengths and the block table are also returned as numpy arrays under ``host``.
     """
     import torch
 
@@ -255,29 +256,46 @@ def make_inputs_device(w: Workload, device, seed: Optional[int] = None) -> Dict[
         return out
 
     block_table = None
+    nan = float("nan")
     if w.paged:
         bs = w.block_size
         max_blocks = (s_max + bs - 1) // bs
         num_blocks = b * max_blocks
         block_table = rng.permutation(num_blocks).astype(np.int32).reshape(b, max_blocks)
+        bt = torch.from_numpy(block_table.astype(np.int64)).to(device)
         if not w.positional:
             # the pool is i.i.d. noise, so drawing it in pool order is the same distribution as
             # drawing per sequence and scattering through the table
             k_cache = draw(b).reshape(num_blocks, bs, hkv, d)
             v_cache = draw(b).reshape(num_blocks, bs, hkv, d)
         else:
-            bt = torch.from_numpy(block_table.astype(np.int64)).to(device)
             k_cache = torch.empty((num_blocks, bs, hkv, d), device=device, dtype=torch.bfloat16)
             v_cache = torch.empty_like(k_cache)
             for i in range(b):
                 k_cache[bt[i]] = draw(1).reshape(max_blocks, bs, hkv, d)
                 v_cache[bt[i]] = draw(1).reshape(max_blocks, bs, hkv, d)
+        if poison:
+            # tokens at positions >= seq_len: the tail of the block that holds position seq_len,
+            # then every later block of the request (one masked fill per request and cache)
+            for i in range(b):
+                n = int(seq_len[i])
+                first, within = divmod(n, bs)
+                for cache in (k_cache, v_cache):
+                    if within and first < max_blocks:
+                        cache[bt[i, first], within:] = nan
+                    lo = first + (1 if within else 0)
+                    if lo < max_blocks:
+                        cache[bt[i, lo:]] = nan
         strides = (bs * row, row, d)
     elif w.share_cache:
         k_cache, v_cache = draw(1), draw(1)
         strides = (0, row, d)
     else:
         k_cache, v_cache = draw(b), draw(b)
+        if poison:
+            for i in range(b):
+                k_cache[i, int(seq_len[i]):] = nan
+                v_cache[i, int(seq_len[i]):] = nan
         strides = (s_max * row, row, d)
 
     return {

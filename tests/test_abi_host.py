@@ -84,6 +84,8 @@ def test_argument_validation_on_host(dsa):
     assert _plan(dsa, _problem(dsa, stride_token=100))[0] == -1
     assert _plan(dsa, _problem(dsa, stride_head=12))[0] == -1
     assert _plan(dsa, _problem(dsa, dtype=7))[0] == -2
+    assert _plan(dsa, _problem(dsa, plan_flags=0x80000000))[0] == -1              # unknown planner switch
+    assert _plan(dsa, _problem(dsa, plan_flags=dsa.DSA_PLAN_NO_ITEM_WARPS))[0] == 0
     assert _plan(dsa, _problem(dsa, block_table=0x30000, block_size=16, max_blocks=10, num_blocks=99))[0] == -1
     assert _plan(dsa, _problem(dsa), _diag(dsa, n_att=2000))[0] == -1
     assert _plan(dsa, _problem(dsa), _diag(dsa, window=0))[0] == -1

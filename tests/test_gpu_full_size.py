@@ -1,6 +1,7 @@
 """Parity at the benchmark's full size and launch configuration: the paged throughput workload
-at batch 256 (18 GB of K/V drawn on the device), checked on sampled requests that the oracle
-computes one by one from a host copy of just their blocks."""
+at batch 32, 128 and 256 (up to 18 GB of K/V drawn on the device, rows past each request's length
+NaN-filled), checked on sampled requests that the oracle computes one by one from a host copy of
+just their blocks, plus the kept-count closed form on every request."""
 import numpy as np
 import pytest
 import torch
@@ -12,12 +13,14 @@ from tests import util
 pytestmark = pytest.mark.gpu
 
 
-def test_config5_batch256_sampled_requests():
+@pytest.mark.parametrize("batch", [32, 128, 256])
+def test_config5_large_batches_sampled_requests(batch):
+    """The paged sweep at batch 32, 128 and 256 (batch 1 and 8 are compared in full elsewhere)."""
     from paper_2609_19702_b200 import binding as dsa
     free, _ = torch.cuda.mem_get_info()
-    if free < 24 << 30:
-        pytest.skip("needs 24 GB of free device memory")
-    w = synth.workload(5, batch=256)
+    if free < (24 << 30) * batch // 256 + (2 << 30):
+        pytest.skip("needs %d GB of free device memory" % (24 * batch // 256 + 2))
+    w = synth.workload(5, batch=batch)
     dev = synth.make_inputs_device(w, torch.device("cuda"))
     prob = dsa.Problem(q=dev["q"], k_cache=dev["k_cache"], v_cache=dev["v_cache"], strides=dev["strides"],
                        seq_len=dev["seq_len"], prompt_len=dev["prompt_len"], num_kv_heads=w.num_kv_heads,
@@ -29,7 +32,7 @@ def test_config5_batch256_sampled_requests():
     order = np.argsort(pos)
     sample = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]),
                      int(np.argmin(np.abs(pos - 208))), int(np.argmin(np.abs(pos - 512))),
-                     int(np.argmin(np.abs(pos - 1024))), 0, 17, 101, 255})
+                     int(np.argmin(np.abs(pos - 1024))), 0, 17 % batch, 101 % batch, batch - 1})
     sub = synth.host_subset(dev, sample)
     out, lse = dsa.alloc_outputs(prob)
     sidx = torch.tensor(sample, device="cuda")
@@ -54,6 +57,8 @@ def test_config5_batch256_sampled_requests():
         # property that holds for every request: kept count = prompt + min(p, N_att) (or p)
         want = w.prompt_len + (pos if diag is None else np.minimum(pos, diag.n_att))
         assert np.array_equal(cnt.cpu().numpy()[:, 0], want)
+    if batch != 256:
+        return
     # the end-to-end call of the benchmark at this size (step inputs and results in pinned host
     # memory): bit for bit what the device-buffer call gives
     diag = dsa.Diag(dsa.DSA_MASK_GRID, 512, 208, w.grid_w, w.row_extra)

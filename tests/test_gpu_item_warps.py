@@ -6,8 +6,6 @@ matches the oracle (kept sets are untouched by it), requests so short that some 
 get no tile at all are handled, and the result -- the entries picked by the fused selection
 included, which the selection tests pin to the oracle on the one-warp plan -- agrees with the
 one-warp-per-item plan of the same library within the summation-order difference."""
-import os
-
 import numpy as np
 import pytest
 import torch
@@ -68,33 +66,29 @@ def test_requests_shorter_than_one_tile_per_warp(dsa):
 def test_shared_item_path_agrees_with_one_warp_per_item(dsa, name, make, splits):
     w = make()
     inp = synth.make_inputs(w)
-    prob = dsa.problem_from_host(inp)
     rng = np.random.default_rng(4)
     trace = synth.random_valid_trace(rng, w.window, w.n_att, (w.batch, w.num_q_heads))
     results = {}
     for setting in ("1", "0"):
-        os.environ["DSA_ITEM_WARPS"] = setting
-        try:
-            outs = []
-            for diag in (None, dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra),
-                         dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att,
-                                  skip_offsets=torch.from_numpy(trace.copy()).cuda(), select=True)):
-                plan = dsa.dsa_query_plan(prob, diag)
-                if diag is not None:
-                    assert plan.item_warps == (4 if setting == "1" else 1), name
-                    if setting == "1":
-                        assert plan.n_split == splits, name
-                out, lse = dsa.alloc_outputs(prob)
-                ws = dsa.alloc_workspace(prob, diag)
-                if diag is None:
-                    dsa.dsa_decode_attention_dense(prob, out, lse, ws)
-                else:
-                    dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
-                torch.cuda.synchronize()
-                outs.append((out.float().cpu(), lse.cpu(), None if diag is None else diag.skip_offsets))
-            results[setting] = outs
-        finally:
-            os.environ.pop("DSA_ITEM_WARPS", None)
+        prob = dsa.problem_from_host(inp, plan_flags=0 if setting == "1" else dsa.DSA_PLAN_NO_ITEM_WARPS)
+        outs = []
+        for diag in (None, dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra),
+                     dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att,
+                              skip_offsets=torch.from_numpy(trace.copy()).cuda(), select=True)):
+            plan = dsa.dsa_query_plan(prob, diag)
+            if diag is not None:
+                assert plan.item_warps == (4 if setting == "1" else 1), name
+                if setting == "1":
+                    assert plan.n_split == splits, name
+            out, lse = dsa.alloc_outputs(prob)
+            ws = dsa.alloc_workspace(prob, diag)
+            if diag is None:
+                dsa.dsa_decode_attention_dense(prob, out, lse, ws)
+            else:
+                dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+            torch.cuda.synchronize()
+            outs.append((out.float().cpu(), lse.cpu(), None if diag is None else diag.skip_offsets))
+        results[setting] = outs
     for (o1, l1, t1), (o0, l0, t0) in zip(results["1"], results["0"]):
         assert torch.allclose(o1, o0, atol=2e-2, rtol=2e-2)
         assert torch.allclose(l1, l0, atol=1e-4, rtol=0)
@@ -113,15 +107,12 @@ def test_shallow_ring_form_matches_the_oracle(dsa):
     plan = _plan(dsa, inp, grid)
     assert plan.stages == 2 and plan.item_warps == 1 and plan.n_split == 1
     _check_all_modes(dsa, inp, list_heads=(1,), seed=5, what="shallow ring, chosen")
-    os.environ["DSA_MMA_STAGES"] = "2"
-    try:
-        for make in (lambda: synth.workload(5, batch=3), lambda: synth.workload(2, batch=8)):
-            w2 = make()
-            inp2 = synth.make_inputs(w2)
-            prob = dsa.problem_from_host(inp2, split_tokens=0)
-            g2 = dsa.Diag(dsa.DSA_MASK_GRID, w2.window, w2.n_att, w2.grid_w, w2.row_extra)
-            if w2.num_kv_heads % 2 == 0 and dsa.dsa_query_plan(prob, g2).item_warps == 1:
-                assert dsa.dsa_query_plan(prob, g2).stages == 2
-            _check_all_modes(dsa, inp2, list_heads=(1,), seed=6, what="shallow ring, forced")
-    finally:
-        os.environ.pop("DSA_MMA_STAGES", None)
+    for make in (lambda: synth.workload(5, batch=3), lambda: synth.workload(2, batch=8)):
+        w2 = make()
+        inp2 = synth.make_inputs(w2)
+        prob = dsa.problem_from_host(inp2, split_tokens=0, plan_flags=dsa.DSA_PLAN_RING_SHALLOW)
+        g2 = dsa.Diag(dsa.DSA_MASK_GRID, w2.window, w2.n_att, w2.grid_w, w2.row_extra)
+        if w2.num_kv_heads % 2 == 0 and dsa.dsa_query_plan(prob, g2).item_warps == 1:
+            assert dsa.dsa_query_plan(prob, g2).stages == 2
+        _check_all_modes(dsa, inp2, list_heads=(1,), seed=6, what="shallow ring, forced",
+                         plan_flags=dsa.DSA_PLAN_RING_SHALLOW)

@@ -33,11 +33,11 @@ def _run_gpu(dsa, prob, diag):
 
 
 def _check_all_modes(dsa, inp, *, f32=False, split_tokens=0, list_heads=(1,), seed=0, what="",
-                     max_prompt_len=None):
+                     max_prompt_len=None, plan_flags=0):
     """Dense, window-only, grid and list masks of one host batch against the oracle."""
     w = inp["workload"]
     dtype = torch.float32 if f32 else torch.bfloat16
-    prob = dsa.problem_from_host(inp, dtype=dtype, split_tokens=split_tokens)
+    prob = dsa.problem_from_host(inp, dtype=dtype, split_tokens=split_tokens, plan_flags=plan_flags)
     if max_prompt_len is not None:
         prob.max_prompt_len = max_prompt_len
     s_max = inp["max_seq_len"]

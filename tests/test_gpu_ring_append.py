@@ -229,3 +229,47 @@ def test_host_io_call_matches_device_call(dsa):
         torch.cuda.synchronize()
         assert torch.equal(h_out.view(torch.int16), ref_out.cpu().view(torch.int16))
         assert torch.equal(h_lse, ref_lse.cpu())
+
+
+def test_prompt_length_above_its_bound_stays_inside_the_request_region(dsa):
+    """A device prompt_len[b] above max_prompt_len is read as max_prompt_len when the cache is a
+    ring: append, fused step and attention then touch only the request's own
+    max_prompt_len + ring_sinks + ring_size tokens (wrong numbers for that request, but no row
+    of a neighbour or beyond the allocation)."""
+    b, h, d, l_p, ring, sinks = 4, 4, 64, 5, 16, 2
+    cap = l_p + sinks + ring
+    row = h * d
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    # one spare region behind the last request as a guard
+    kc = torch.randn(((b + 1) * cap, h, d), generator=gen, device="cuda").to(torch.bfloat16)
+    vc = torch.randn(((b + 1) * cap, h, d), generator=gen, device="cuda").to(torch.bfloat16)
+    q = torch.randn((b, h, d), generator=gen, device="cuda").to(torch.bfloat16)
+    k_new, v_new = q.clone() + 1, q.clone() - 1
+    seq = torch.tensor([60, 70, 23, 40], dtype=torch.int32, device="cuda")
+    bad_prompt = torch.tensor([5, 12, 5, 23], dtype=torch.int32, device="cuda")     # two of them above the bound of 5
+    prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d), seq_len=seq,
+                       prompt_len=bad_prompt, num_kv_heads=h, max_seq_len=100, max_prompt_len=l_p,
+                       ring_size=ring, ring_sinks=sinks)
+    diag = dsa.Diag(dsa.DSA_MASK_GRID, ring, 6, 5, 0, n_sink=sinks)
+    out, lse = dsa.alloc_outputs(prob)
+    ws = dsa.alloc_workspace(prob, diag)
+
+    def changed_rows(before_k, before_v):
+        ck = (kc.view(torch.int16) != before_k).any(dim=2).any(dim=1)
+        cv = (vc.view(torch.int16) != before_v).any(dim=2).any(dim=1)
+        assert torch.equal(ck, cv)
+        return torch.nonzero(ck).flatten().tolist()
+
+    for fused in (False, True):
+        bk, bv = kc.view(torch.int16).clone(), vc.view(torch.int16).clone()
+        if fused:
+            dsa.dsa_decode_step(prob, diag, k_new, v_new, out, lse, ws)
+        else:
+            dsa.dsa_append_kv(prob, k_new, v_new, advance=False)
+            dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws)
+        torch.cuda.synchronize()
+        rows = changed_rows(bk, bv)
+        assert len(rows) == b and [r // cap for r in rows] == list(range(b)), rows   # one row per request, in its own region
+        assert torch.isfinite(out.float()).all()
+        k_new, v_new = k_new + 1, v_new + 1

@@ -8,7 +8,9 @@ although the array still holds the previous call's partials."""
 import pytest
 import torch
 
+from oracle import oracle as ora
 from paper_2609_19702_b200 import synth
+from tests import util
 
 pytestmark = pytest.mark.gpu
 
@@ -34,9 +36,12 @@ def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row():
         return out.float(), lse
 
     ref_dense, ref_sparse = reference(None), reference(diag)
+    # what the paper's definitions give for the same batch (float64 oracle)
+    ora_dense = util.oracle_run(inp, ora.MODE_DENSE)
+    ora_sparse = util.oracle_run(inp, ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride=w.stride)
     # two calls in a row, alternating problems so that each sees the other's leftovers
     for _ in range(2):
-        for dg, (ref_out, ref_lse) in ((None, ref_dense), (diag, ref_sparse)):
+        for dg, (ref_out, ref_lse), ora_ref in ((None, ref_dense, ora_dense), (diag, ref_sparse, ora_sparse)):
             out, lse = dsa.alloc_outputs(prob)
             out.fill_(float("nan"))
             lse.fill_(float("nan"))
@@ -45,6 +50,7 @@ def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row():
             err = (out.float() - ref_out).abs() - (1e-2 + 1e-2 * ref_out.abs())
             assert torch.isfinite(out.float()).all() and err.max().item() <= 0
             assert (lse - ref_lse).abs().max().item() <= 1e-3
+            util.assert_close(out, lse, ora_ref, what="static scratch against the oracle")
 
     # a problem whose partials do not fit the fixed array is refused, nothing is launched
     big = synth.workload(5, batch=256)
