@@ -275,14 +275,18 @@ def time_flushed(torch, fn, flush, iters=30, warmup=3):
     return float(np.median(times)), float(np.min(times))
 
 
-def per_config_table(torch, dsa, synth, dev, peak):
-    """Every configuration, dense and sparse from the same library, one call at a time."""
+def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
+    """Every configuration, dense and sparse from the same library, one call at a time.
+    plan_flags: planner switches for comparison runs (0: the library chooses); only: restrict to
+    these (config, batch) pairs."""
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     rows = []
     todo = [(synth.workload(i), None) for i in (1, 2, 3, 4)]
     for b in (1, 8, 32, 128, 256):
         todo.append((synth.workload(5, batch=b), [(512, 208), (1024, 416)]))
     for w, windows in todo:
+        if only is not None and (w.index, w.batch) not in only:
+            continue
         inputs = synth.make_inputs_device(w, dev)
         host = inputs["host"]
         prob = dsa.Problem(
@@ -290,7 +294,8 @@ def per_config_table(torch, dsa, synth, dev, peak):
             seq_len=inputs["seq_len"], prompt_len=inputs["prompt_len"], num_kv_heads=w.num_kv_heads,
             max_seq_len=inputs["max_seq_len"], max_prompt_len=w.prompt_len,
             block_table=inputs["block_table"], block_size=inputs["block_size"],
-            num_blocks=0 if inputs["block_table"] is None else inputs["block_table"].numel())
+            num_blocks=0 if inputs["block_table"] is None else inputs["block_table"].numel(),
+            plan_flags=plan_flags)
         out, lse = dsa.alloc_outputs(prob)
         ws = dsa.alloc_workspace(prob, None)
         plan = dsa.dsa_query_plan(prob, None)
@@ -384,7 +389,8 @@ def mask_variants(torch, dsa, synth, dev, peak):
 
 
 def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
-                      modes=("dense", "sparse", "sparse_select", "dense_two_calls", "sparse_two_calls")):
+                      modes=("dense", "sparse", "sparse_select", "dense_two_calls", "sparse_two_calls"),
+                      plan_flags=0):
     """Whole-image decode loop: 1024 image tokens after a 50-token prompt, `batch` requests (16: the
     shape of the paper's Lumina-mGPT latency runs), 32/32 heads, head_dim 128, over `n_layers`
     layers, each with its own KV cache (together larger than the L2).  Every step appends the new
@@ -421,7 +427,7 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
             pl = torch.full((b,), l_p, dtype=torch.int32, device=dev)
             prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d),
                                seq_len=seq, prompt_len=pl, num_kv_heads=h, max_seq_len=s_max,
-                               max_prompt_len=l_p, ring_size=ring)
+                               max_prompt_len=l_p, ring_size=ring, plan_flags=plan_flags)
             out, lse = dsa.alloc_outputs(prob)
             ldiag = diag
             if kind == "sparse_select":
@@ -479,7 +485,7 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
         res[mode] = {"ms_per_image": round(best, 3), "us_per_step": round(best / steps * 1e3, 2),
                      "us_per_layer_step": round(best / steps / n_layers * 1e3, 2),
                      "us_last_step": round(last / reps * 1e3, 2), "cache_GB": round(cache_gb, 3),
-                     "n_split": plan.n_split,
+                     "n_split": plan.n_split, "heads_per_block": plan.heads_per_block,
                      "launches_per_layer_step": plan.launches + (0 if fused else 1)}
         del layers, graph
         torch.cuda.empty_cache()
@@ -746,7 +752,8 @@ def run_ours(args):
                                 "grid_blocks": plan.grid_blocks, "smem_bytes": plan.smem_bytes,
                                 "tile_tokens": plan.tile_tokens, "stages": plan.stages,
                                 "tensor_cores": plan.tensor_cores, "work_items": plan.work_items,
-                                "item_warps": plan.item_warps}},
+                                "item_warps": plan.item_warps, "heads_per_block": plan.heads_per_block,
+                                "block_warps": plan.block_warps}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }

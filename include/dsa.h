@@ -130,6 +130,11 @@ typedef struct dsa_problem {
 #define DSA_PLAN_NO_ITEM_WARPS 0x02u  /* small launches: split + combine, never four warps on one item   */
 #define DSA_PLAN_RING_DEEP     0x04u  /* two-heads-per-block kernel: keep the 3-stage ring               */
 #define DSA_PLAN_RING_SHALLOW  0x08u  /* two-heads-per-block kernel: take the 2-stage ring               */
+#define DSA_PLAN_GROUP         0x10u  /* take the head-group kernel wherever it can run                  */
+#define DSA_PLAN_NO_GROUP      0x20u  /* never take the head-group kernel                                */
+#define DSA_PLAN_GROUP_W4      0x40u  /* forced head-group kernel: 4 warps per block instead of 2        */
+#define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
+#define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u
 
 /*
  * Which decode keys are kept (Algorithm 1 with its data-dependent selection made an input).
@@ -197,6 +202,10 @@ typedef struct dsa_plan_info {
     int32_t work_items;     /* (request, kv head, split) items                                     */
     int32_t item_warps;     /* warps that share one work item (4 in small tensor-core launches,    */
                             /* merged in shared memory; else 1)                                    */
+    int32_t heads_per_block;/* head-group tensor-core kernel: kv heads that share the one row list */
+                            /* a block builds (its warps stream heads_per_block / block_warps      */
+                            /* heads each, back to back); 0: another kernel                        */
+    int32_t block_warps;    /* warps per thread block                                              */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);

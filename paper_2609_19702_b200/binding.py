@@ -21,6 +21,15 @@ DSA_BF16, DSA_F32 = 0, 1
 DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
 # dsa_problem.plan_flags: 0 lets the library plan; the bits force single decisions (comparison runs, tests)
 DSA_PLAN_CUDA_CORES, DSA_PLAN_NO_ITEM_WARPS, DSA_PLAN_RING_DEEP, DSA_PLAN_RING_SHALLOW = 0x1, 0x2, 0x4, 0x8
+DSA_PLAN_GROUP, DSA_PLAN_NO_GROUP, DSA_PLAN_GROUP_W4 = 0x10, 0x20, 0x40
+DSA_PLAN_HEADS_PER_WARP_SHIFT = 8
+
+
+def plan_group(warps: int, heads_per_warp: int) -> int:
+    """plan_flags that force the head-group kernel with `warps` (2 or 4) warps per block, each
+    streaming `heads_per_warp` kv heads."""
+    assert warps in (2, 4) and 1 <= heads_per_warp <= 255
+    return DSA_PLAN_GROUP | (DSA_PLAN_GROUP_W4 if warps == 4 else 0) | (heads_per_warp << DSA_PLAN_HEADS_PER_WARP_SHIFT)
 
 EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_workspace_size",
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
@@ -58,7 +67,8 @@ class dsa_plan_info(ctypes.Structure):
                 ("launches", ctypes.c_int32), ("grid_blocks", ctypes.c_int32),
                 ("smem_bytes", ctypes.c_int32), ("tile_tokens", ctypes.c_int32),
                 ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32),
-                ("item_warps", ctypes.c_int32)]
+                ("item_warps", ctypes.c_int32), ("heads_per_block", ctypes.c_int32),
+                ("block_warps", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:

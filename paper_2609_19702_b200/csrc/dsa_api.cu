@@ -42,8 +42,9 @@ int sm_count() {
     return n;
 }
 
-constexpr uint32_t kKnownPlanFlags =
-    DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_RING_DEEP | DSA_PLAN_RING_SHALLOW;
+constexpr uint32_t kKnownPlanFlags = DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_RING_DEEP |
+                                     DSA_PLAN_RING_SHALLOW | DSA_PLAN_GROUP | DSA_PLAN_NO_GROUP |
+                                     DSA_PLAN_GROUP_W4 | DSA_PLAN_HEADS_PER_WARP_MASK;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -62,6 +63,10 @@ struct Plan {
     int mma_warps;       // warps (= kv heads) per block that share one row list
     int mma_kw;          // warps that share one work item (small launches), 1 or kMmaItemWarps
     int mma_stages;      // ring depth of the tensor-core kernel
+    int group_w;         // head-group tensor-core kernel: warps per block (0: not that kernel)
+    int group_u;         // and kv heads each warp streams through the block's one row list
+    int group_stages;    // and its ring depth
+    int64_t blocks;      // its grid
     int64_t grid;
     size_t smem;
     size_t ws_out_bytes, ws_lse_bytes, ws_sel_bytes, ws_total;
@@ -85,6 +90,7 @@ KernelQuery kernel_query(const Plan& pl) {
     KernelQuery q;
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
     q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
+    q.group_w = pl.group_w; q.group_stages = pl.group_stages;
     return q;
 }
 
@@ -146,6 +152,61 @@ int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
 
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
+// How many kv heads each warp of the head-group kernel should stream (a power of two), and with which
+// ring depth.
+//
+// Measured on the paged workload (window 512 / N_att 208, 32 kv heads, W = 4, 296 blocks resident) and
+// on the decode-loop shape (50 prompt tokens + N_att 52): whatever the batch, the best U is the one
+// that makes the grid JUST FIT the device -- 0.86 of a wave at batch 32 / 64 / 128 / 256 with
+// U = 1 / 2 / 4 / 8 (37 / 68 / 130 / 256 us against 39 / 72 / 142 / 268 us for two heads per block;
+// decode loop at batch 64 / 128 / 256: 22.5 / 40.3 / 75.8 us against 24.9 / 47.9 / 85.2 us).  Every
+// block is then resident from the start and every warp streams U heads without a block turning
+// over.  A grid of 1.3 waves is the worst case (+25 %), 1.7 and 3.5 waves cost 5-10 %, and under one
+// wave the time is that of one block: at half a wave a larger U doubles it.  The estimate below is
+// that table: (list building + U heads of `tiles` tiles) x (waves, a partial one counted half-way
+// between its size and a whole one) x (time per tile, which grows with the warps that share an SM).
+// The shallow ring (one tile in flight per warp instead of two, about 3 % slower when the grid
+// fits either way) holds half as many blocks again per SM: it is for grids that would otherwise
+// spill a little into a second wave (batch 40: 46 us against 55 us).
+// Split plans keep U = 1: most of their (request, split) blocks are empty or short, the real wave
+// count is unknown, and long blocks make a long tail (dense, batch 256: 1380 us at U = 1, 1516 at U = 8).
+int choose_heads_per_warp(const dsa_problem* p, const Plan& pl, int w, int64_t bound, size_t smem_deep,
+                          size_t smem_shallow, int num_sms, int* stages) {
+    const bool want_shallow = (p->plan_flags & DSA_PLAN_RING_SHALLOW) != 0 && smem_shallow != 0;
+    const bool want_deep = (p->plan_flags & DSA_PLAN_RING_DEEP) != 0 && !want_shallow;
+    *stages = want_shallow ? kGroupStagesShallow : kGroupStages;
+    if (pl.n_split > 1) return 1;
+    const double tiles = std::max(1.0, (double)bound / std::max(pl.tile, 1));
+    const double build = 3.0;                              // list building, in units of one 16-key tile
+    int best = 0;
+    double best_cost = 0;
+    for (int shallow = 0; shallow < 2; ++shallow) {
+        const size_t smem = shallow ? smem_shallow : smem_deep;
+        if (shallow ? (smem == 0 || want_deep) : want_shallow) continue;
+        const int64_t per_sm = std::max<int64_t>(1, (int64_t)(228 * 1024) / (int64_t)(smem + 1024));
+        const double slots = (double)per_sm * num_sms;
+        for (int u = 1; u * w <= p->num_kv_heads; u *= 2) {
+            if (p->num_kv_heads % (u * w)) break;
+            const double blocks = (double)p->batch * (p->num_kv_heads / (u * w));
+            const double waves = blocks / slots;
+            const double block_time = build + u * tiles;
+            // how long a warp takes per tile depends on how many warps share its SM: 8 (the deep ring,
+            // full) is the unit; fewer run up to a third faster, the shallow ring's 12 run 1.55 x slower
+            const double full = (double)per_sm * w / 8.0;
+            const double load = std::min(waves, 1.0) * full;
+            const double per_tile = load <= 1.0 ? 0.67 + 0.33 * load : 1.0 + 1.1 * (load - 1.0);
+            double cost = block_time * per_tile;
+            if (waves > 1.0) cost *= waves * (1.0 + 0.5 * std::max(0.0, std::ceil(waves - 0.05) / waves - 1.0));
+            if (shallow) cost *= 1.02;
+            if (best == 0 || cost < best_cost * 1.005) {    // (ties go to the larger U: a grid that just fits has no turnover)
+                best = u; best_cost = cost;
+                *stages = shallow ? kGroupStagesShallow : kGroupStages;
+            }
+        }
+    }
+    return std::max(best, 1);
+}
+
 int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     int32_t rc = check_problem(p);
     if (rc != DSA_OK) return rc;
@@ -178,6 +239,10 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->mma_warps = 1;
     pl->mma_kw = 1;
     pl->mma_stages = kMmaStages;
+    pl->group_w = 0;
+    pl->group_u = 0;
+    pl->group_stages = kGroupStages;
+    pl->blocks = 0;
     if (pl->mma) {
         const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
         // two kv heads per block (measured: 2 beats 1 and 4) when the row list can be shared
@@ -222,7 +287,9 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         // 32.8 us against 29.7 us for three splits and the combine; with ~1000-row items the
         // single launch still wins there).  Requests beyond 2048 rows need the combine anyway;
         // there the merge on top of it measured as a small loss.
-        if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK && !(p->plan_flags & DSA_PLAN_NO_ITEM_WARPS)) {
+        // (a forced head-group kernel takes the place of the small-launch form as well)
+        if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK &&
+            !(p->plan_flags & (DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_GROUP))) {
             const int64_t kw_blocks = pairs * ((want_split + kMmaItemWarps - 1) / kMmaItemWarps);
             if (kw_blocks <= 2 * kNumSMs || kw_blocks >= 4 * kNumSMs || bound > MAX_CHUNK) {
                 pl->mma_kw = kMmaItemWarps;
@@ -246,8 +313,47 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->grid = (int64_t)p->batch * p->num_kv_heads * pl->n_split;
     if (pl->grid > 0x7fffffffLL) return DSA_ERR_UNSUPPORTED;
 
+    // Head-group form: one row list per (request, split), built by a block of W warps and streamed by
+    // each of them for U kv heads back to back.  Needs a mask that does not depend on the head.
+    // With U = 1 it performs like the two-heads-per-block kernel (22.2 / 37.4 / 70.1 / 140 / 263 us
+    // against 22.6 / 39.0 / 72.4 / 142 / 268 us on the paged workload at batch 16 ... 256); larger U
+    // amortise the list over more heads and, more important, let the planner make the grid just
+    // fit the device (see choose_heads_per_warp).
+    if (pl->mma && pl->mma_kw == 1 && !(p->plan_flags & DSA_PLAN_NO_GROUP)) {
+        const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
+        const bool forced = (p->plan_flags & DSA_PLAN_GROUP) != 0;
+        const int w = forced ? ((p->plan_flags & DSA_PLAN_GROUP_W4) ? 4 : 2) : 4;
+        if (shared_mask && p->num_kv_heads % w == 0) {
+            int u = (int)((p->plan_flags & DSA_PLAN_HEADS_PER_WARP_MASK) >> DSA_PLAN_HEADS_PER_WARP_SHIFT);
+            int stages = (p->plan_flags & DSA_PLAN_RING_SHALLOW) ? kGroupStagesShallow : kGroupStages;
+            if (!forced || u < 1) {
+                Plan probe = *pl;
+                probe.group_w = w;
+                KernelShape gs[2] = {};
+                int32_t rcg = DSA_OK;
+                for (int sh = 0; sh < 2 && rcg == DSA_OK; ++sh) {
+                    probe.group_stages = sh ? kGroupStagesShallow : kGroupStages;
+                    rcg = dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
+                        using T = decltype(t);
+                        return kernel_shape<T, decltype(dd)::value>(kernel_query(probe), pl->chunk, pl->bitmap_words, &gs[sh])
+                                   ? DSA_OK : DSA_ERR_UNSUPPORTED;
+                    });
+                }
+                u = rcg == DSA_OK ? choose_heads_per_warp(p, *pl, w, bound, gs[0].smem, gs[1].smem, kNumSMs, &stages) : 0;
+            }
+            if (u >= 1 && p->num_kv_heads % (w * u) == 0) {
+                pl->group_w = w;
+                pl->group_u = u;
+                pl->group_stages = stages;
+                pl->mma_warps = 1;
+                pl->blocks = (int64_t)p->batch * pl->n_split * (p->num_kv_heads / (w * u));
+            }
+        }
+    }
     rc = shape_of(pl->chunk, &shape);                         // (the small-launch form may have been chosen since)
     if (rc != DSA_OK) return rc;
+    pl->stages = shape.stages;
+
     // Ring depth of the two-heads-per-block kernel.  Shared memory decides how many blocks an SM
     // holds, and a launch of a few waves pays for every block beyond a whole number of them: a
     // last wave costs at least about half a full one, however few blocks it has (measured on the
@@ -260,7 +366,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     // loss of 10 % on the dense calls at batch 1-8).
     const bool force_shallow = (p->plan_flags & DSA_PLAN_RING_SHALLOW) != 0;
     const bool force_deep = (p->plan_flags & DSA_PLAN_RING_DEEP) != 0 && !force_shallow;
-    if (pl->mma && pl->mma_warps == 2 && pl->mma_kw == 1 && p->split_tokens == 0 &&
+    if (pl->mma && pl->group_w == 0 && pl->mma_warps == 2 && pl->mma_kw == 1 && p->split_tokens == 0 &&
         (pl->n_split == 1 || force_shallow) && !force_deep) {
         Plan alt = *pl;
         alt.mma_stages = kMmaStagesShallow;
@@ -337,6 +443,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.trace_len = (d && pl.mode == MODE_LIST) ? d->trace_len : 0;
     a->mask.bitmap_words = pl.bitmap_words;
     a->chunk = pl.chunk; a->n_split = pl.n_split;
+    a->heads_per_warp = pl.group_u;
     a->n_items = (int)pl.grid;
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
@@ -428,7 +535,8 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     cudaError_t err = cudaSuccess;
     rc = dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
         using T = decltype(t);
-        err = kernel_launch<T, decltype(dd)::value>(kernel_query(pl), step && pl.mma, a, pl.grid, pl.smem, st);
+        err = kernel_launch<T, decltype(dd)::value>(kernel_query(pl), step && pl.mma, a, pl.grid, pl.smem, st,
+                                                    pl.blocks);
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;
@@ -510,7 +618,9 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->split_tokens = pl.chunk;
     info->n_split = pl.n_split;
     info->launches = problem->batch == 0 ? 0 : (pl.n_split > 1 ? 2 : 1);
-    info->grid_blocks = (int32_t)(pl.mma ? pl.grid / pl.mma_warps : pl.grid);
+    info->grid_blocks = (int32_t)(pl.group_w > 0 ? pl.blocks : (pl.mma ? pl.grid / pl.mma_warps : pl.grid));
+    info->heads_per_block = pl.group_w * pl.group_u;
+    info->block_warps = pl.mma ? (pl.group_w > 0 ? pl.group_w : pl.mma_warps * pl.mma_kw) : 4;
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;
     info->tensor_cores = pl.mma ? 1 : 0;

@@ -29,6 +29,7 @@ struct AttnArgs {
     int B, H_q, H_kv;
     float scale_log2;            // sm_scale * log2(e)
     MaskArgs mask;
+    int heads_per_warp;          // head-group kernel: kv heads each warp streams back to back through one row list
     int chunk;                   // kept rows per split (multiple of the tile; see MAX_CHUNK)
     int n_split;
     int n_items;                 // B * H_kv * n_split work items

@@ -3,6 +3,7 @@
 #pragma once
 #include "dsa_attn.cuh"
 #include "dsa_attn_mma.cuh"
+#include "dsa_attn_group.cuh"
 #include "dsa_launch.cuh"
 
 #include <atomic>
@@ -80,6 +81,41 @@ struct KernelPick {
         if (e != cudaSuccess) return e;
         return launch_pdl(kern, (unsigned)grid, 32 * W * KW, smem_bytes, st, a);
     }
+    // Head-group tensor-core kernel (bf16, masks that do not depend on the head): blocks of W warps,
+    // one row list per block; rings of kGroupStages slots, or kGroupStagesShallow for more blocks per SM.
+    template <int W, int ST>
+    static size_t smem_group_w(int chunk, int bw) { return GroupCfg<D, W, ST>::smem_bytes(chunk, bw); }
+    static size_t smem_group(int w, int stages, int chunk, int bw) {
+        if (stages == kGroupStagesShallow)
+            return w == 4 ? smem_group_w<4, kGroupStagesShallow>(chunk, bw) : smem_group_w<2, kGroupStagesShallow>(chunk, bw);
+        return w == 4 ? smem_group_w<4, kGroupStages>(chunk, bw) : smem_group_w<2, kGroupStages>(chunk, bw);
+    }
+    template <int W, bool APPEND, int ST>
+    static ConfiguredFlags* group_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    template <int W, bool APPEND, int ST>
+    static cudaError_t launch_group_w(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
+        if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            auto kern = dsa_attn_group_kernel<D, G, ST, W, APPEND>;
+            const cudaError_t e = ensure_configured(kern, group_configured<W, APPEND, ST>());
+            if (e != cudaSuccess) return e;
+            return launch_pdl(kern, (unsigned)blocks, 32 * W, smem_bytes, st, a);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
+    template <int ST>
+    static cudaError_t launch_group_s(int w, bool append, const AttnArgs& a, int64_t blocks, size_t smem_bytes,
+                                      cudaStream_t st) {
+        if (w == 4) return append ? launch_group_w<4, true, ST>(a, blocks, smem_bytes, st)
+                                  : launch_group_w<4, false, ST>(a, blocks, smem_bytes, st);
+        return append ? launch_group_w<2, true, ST>(a, blocks, smem_bytes, st)
+                      : launch_group_w<2, false, ST>(a, blocks, smem_bytes, st);
+    }
+    static cudaError_t launch_group(int w, int stages, bool append, const AttnArgs& a, int64_t blocks,
+                                    size_t smem_bytes, cudaStream_t st) {
+        return stages == kGroupStagesShallow ? launch_group_s<kGroupStagesShallow>(w, append, a, blocks, smem_bytes, st)
+                                             : launch_group_s<kGroupStages>(w, append, a, blocks, smem_bytes, st);
+    }
     // Configure every kernel of this variant for the current device (see dsa_prepare).
     static cudaError_t prepare() {
         cudaError_t e = ensure_configured(dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>, cc_configured());
@@ -101,6 +137,22 @@ struct KernelPick {
             mma(one{}, std::false_type{}, four{}, deep{});
             mma(one{}, std::true_type{}, four{}, deep{});
             if constexpr (!HM && !SEL) {
+                auto group = [&](auto w, auto app, auto stg) {
+                    constexpr int W = decltype(w)::value, ST = decltype(stg)::value;
+                    constexpr bool APPEND = decltype(app)::value;
+                    if (e == cudaSuccess)
+                        e = ensure_configured(dsa_attn_group_kernel<D, G, ST, W, APPEND>, group_configured<W, APPEND, ST>());
+                };
+                using gdeep = std::integral_constant<int, kGroupStages>;
+                using gshallow = std::integral_constant<int, kGroupStagesShallow>;
+                group(two{}, std::false_type{}, gdeep{});
+                group(two{}, std::true_type{}, gdeep{});
+                group(four{}, std::false_type{}, gdeep{});
+                group(four{}, std::true_type{}, gdeep{});
+                group(two{}, std::false_type{}, gshallow{});
+                group(two{}, std::true_type{}, gshallow{});
+                group(four{}, std::false_type{}, gshallow{});
+                group(four{}, std::true_type{}, gshallow{});
                 mma(two{}, std::false_type{}, one{}, deep{});
                 mma(two{}, std::true_type{}, one{}, deep{});
                 mma(two{}, std::false_type{}, one{}, shallow{});
@@ -162,6 +214,11 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
     return dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
         out->tile = q.mma ? MMA_KEYS : P::TILE;
+        if (q.mma && q.group_w > 0) {
+            out->stages = q.group_stages == kGroupStagesShallow ? kGroupStagesShallow : kGroupStages;
+            out->smem = P::smem_group(q.group_w, out->stages, chunk, bitmap_words);
+            return;
+        }
         const bool shallow = q.mma && q.mma_stages == kMmaStagesShallow && q.mma_warps == 2 && q.mma_kw == 1 &&
                              !q.headmask && !q.select;
         out->stages = q.mma ? (shallow ? kMmaStagesShallow : kMmaStages) : P::STAGES;
@@ -172,10 +229,12 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
 
 template <typename T, int D>
 cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
-                          cudaStream_t st) {
+                          cudaStream_t st, int64_t blocks) {
     cudaError_t err = cudaErrorInvalidValue;
     dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
+        if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
+        else
         err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, q.mma_stages, a, items, smem, st, append)
                     : P::launch(a, items, smem, st);
     });

@@ -9,7 +9,11 @@ namespace dsa {
 constexpr int kMaxDevices = 64;
 constexpr int kMmaItemWarps = 4;                   // warps per work item in small launches
 constexpr int kMmaStages = 3;                      // ring slots per warp: two 16-key tiles in flight, one being consumed
-constexpr int kMmaStagesShallow = 2;               // the shallow-ring form of the two-heads-per-block kernel
+constexpr int kMmaStagesShallow = 2;
+constexpr int kGroupStagesShallow = 2;             // shallow form: half as many blocks again per SM
+constexpr int kGroupStages = 3;                    // ring slots per warp of the head-group kernel (4 and 6 slots with
+                                                   // fewer warps per SM measured 25-45 % slower: the warps, not the
+                                                   // bytes in flight, carry the throughput)               // the shallow-ring form of the two-heads-per-block kernel
 
 // Which kernel variant a call needs.
 struct KernelQuery {
@@ -20,6 +24,9 @@ struct KernelQuery {
     int mma_warps;           // tensor-core kernel: kv heads per block that share one row list (1 or 2)
     int mma_kw;              // tensor-core kernel: warps that share one work item (1 or kMmaItemWarps)
     int mma_stages;          // tensor-core kernel: kMmaStages, or kMmaStagesShallow (two heads per block only)
+    int group_w;             // head-group tensor-core kernel: warps per block that share one row list for
+                             // group_w x heads_per_warp kv heads (2 or 4); 0: not that kernel
+    int group_stages;        // its ring depth: kGroupStages or kGroupStagesShallow
 };
 
 struct KernelShape {
@@ -33,10 +40,11 @@ template <typename T, int D>
 bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape* out);
 
 // Launch it: `items` (request, kv head, split) work items; `append`: the fused decode step (the
-// kernel reads the current token's rows from a.k_new / a.v_new and stores them to the cache).
+// kernel reads the current token's rows from a.k_new / a.v_new and stores them to the cache);
+// `blocks`: thread blocks of the head-group kernel (ignored by the others).
 template <typename T, int D>
 cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
-                          cudaStream_t st);
+                          cudaStream_t st, int64_t blocks);
 
 // Configure every variant of (T, D) for the current device, so that no later launch has to (a
 // launch inside a stream capture must not).

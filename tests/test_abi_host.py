@@ -86,6 +86,12 @@ def test_argument_validation_on_host(dsa):
     assert _plan(dsa, _problem(dsa, dtype=7))[0] == -2
     assert _plan(dsa, _problem(dsa, plan_flags=0x80000000))[0] == -1              # unknown planner switch
     assert _plan(dsa, _problem(dsa, plan_flags=dsa.DSA_PLAN_NO_ITEM_WARPS))[0] == 0
+    rc, info = _plan(dsa, _problem(dsa, batch=64, num_q_heads=32, num_kv_heads=32, max_seq_len=4360, max_prompt_len=200,
+                                   plan_flags=dsa.plan_group(4, 2)), _diag(dsa, window=512, n_att=208, grid_w=64))
+    assert rc == 0 and info.heads_per_block == 8 and info.block_warps == 4 and info.grid_blocks == 64 * 4
+    rc, info = _plan(dsa, _problem(dsa, batch=64, num_q_heads=32, num_kv_heads=32, max_seq_len=4360, max_prompt_len=200,
+                                   plan_flags=dsa.DSA_PLAN_NO_GROUP), _diag(dsa, window=512, n_att=208, grid_w=64))
+    assert rc == 0 and info.heads_per_block == 0
     assert _plan(dsa, _problem(dsa, block_table=0x30000, block_size=16, max_blocks=10, num_blocks=99))[0] == -1
     assert _plan(dsa, _problem(dsa), _diag(dsa, n_att=2000))[0] == -1
     assert _plan(dsa, _problem(dsa), _diag(dsa, window=0))[0] == -1
@@ -101,7 +107,11 @@ def test_plan_sizes(dsa):
     rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,
                                    max_prompt_len=200), _diag(dsa, window=512, n_att=208, grid_w=64))
     assert rc == 0 and info.n_split == 1 and info.launches == 1
-    assert info.grid_blocks in (256 * 32, 256 * 16, 256 * 8)     # 1, 2 or 4 kv heads per block
+    if info.heads_per_block:                                     # one row list per block, shared by these heads
+        assert info.grid_blocks * info.heads_per_block == 256 * 32 and info.block_warps in (2, 4)
+        assert info.heads_per_block % info.block_warps == 0
+    else:
+        assert info.grid_blocks in (256 * 32, 256 * 16)          # 1 or 2 kv heads per block
     # dense on the same problem needs splits and the combine kernel
     rc, info = _plan(dsa, _problem(dsa, batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360))
     assert rc == 0 and info.n_split * info.split_tokens >= 4360 and info.launches == 2
