@@ -130,8 +130,8 @@ typedef struct dsa_problem {
 #define DSA_PLAN_NO_ITEM_WARPS 0x02u  /* small launches: split + combine, never four warps on one item   */
 #define DSA_PLAN_RING_DEEP     0x04u  /* two-heads-per-block kernel: keep the 3-stage ring               */
 #define DSA_PLAN_RING_SHALLOW  0x08u  /* two-heads-per-block kernel: take the 2-stage ring               */
-#define DSA_PLAN_GROUP         0x10u  /* take the head-group kernel wherever it can run                  */
-#define DSA_PLAN_NO_GROUP      0x20u  /* never take the head-group kernel                                */
+#define DSA_PLAN_GROUP         0x10u  /* take the head-group / per-head-list kernels wherever they can run */
+#define DSA_PLAN_NO_GROUP      0x20u  /* never take them                                                 */
 #define DSA_PLAN_GROUP_W4      0x40u  /* forced head-group kernel: 4 warps per block instead of 2        */
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u
@@ -206,6 +206,8 @@ typedef struct dsa_plan_info {
                             /* a block builds (its warps stream heads_per_block / block_warps      */
                             /* heads each, back to back); 0: another kernel                        */
     int32_t block_warps;    /* warps per thread block                                              */
+    int32_t per_head_lists; /* 1: the per-head-list tensor-core kernel (list masks per head, fused  */
+                            /* selection): shared tables per block, one candidate list per head    */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);

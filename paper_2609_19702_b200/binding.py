@@ -68,7 +68,7 @@ class dsa_plan_info(ctypes.Structure):
                 ("smem_bytes", ctypes.c_int32), ("tile_tokens", ctypes.c_int32),
                 ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32),
                 ("item_warps", ctypes.c_int32), ("heads_per_block", ctypes.c_int32),
-                ("block_warps", ctypes.c_int32)]
+                ("block_warps", ctypes.c_int32), ("per_head_lists", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:

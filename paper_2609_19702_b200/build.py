@@ -19,12 +19,12 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdsa.so")
 SOURCES = ["dsa_api.cu", "dsa_kernels_bf16_d128.cu", "dsa_kernels_bf16_d64.cu", "dsa_kernels_f32_d128.cu",
            "dsa_kernels_f32_d64.cu"]
-HEADERS = ["dsa_attn.cuh", "dsa_attn_mma.cuh", "dsa_tile.cuh", "dsa_common.cuh", "dsa_mask.cuh", "dsa_launch.cuh",
-           "dsa_kernels.cuh", "dsa_aux.cuh", os.path.join("..", "..", "include", "dsa.h")]
 
 
 def _newest_source_mtime() -> float:
-    paths = [os.path.join(CSRC, s) for s in SOURCES + HEADERS]
+    """Newest of the translation units, every header under csrc/ and the public header."""
+    paths = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h"))]
+    paths.append(os.path.join(HERE, "..", "include", "dsa.h"))
     return max(os.path.getmtime(p) for p in paths if os.path.exists(p))
 
 

@@ -53,6 +53,7 @@ constexpr int kMaxSplits = 8192;                 // split weights of the combine
 // The launch plan: how many kept rows one block takes, how many splits that makes.
 struct Plan {
     int mode;            // MODE_*
+    int window;          // N_r of the sparse call (0: dense)
     int G;
     bool headmask;
     bool select;
@@ -66,6 +67,8 @@ struct Plan {
     int group_w;         // head-group tensor-core kernel: warps per block (0: not that kernel)
     int group_u;         // and kv heads each warp streams through the block's one row list
     int group_stages;    // and its ring depth
+    bool heads;          // per-head-list tensor-core kernel (kHeadsWarps warps per block, group_u heads per warp)
+    int dir_cap, kidx_cap;
     int64_t blocks;      // its grid
     int64_t grid;
     size_t smem;
@@ -91,6 +94,7 @@ KernelQuery kernel_query(const Plan& pl) {
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
     q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
     q.group_w = pl.group_w; q.group_stages = pl.group_stages;
+    q.heads = pl.heads; q.dir_cap = pl.dir_cap; q.kidx_cap = pl.kidx_cap; q.window = pl.window;
     return q;
 }
 
@@ -242,6 +246,9 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->group_w = 0;
     pl->group_u = 0;
     pl->group_stages = kGroupStages;
+    pl->heads = false;
+    pl->dir_cap = pl->kidx_cap = 0;
+    pl->window = d ? d->window : 0;
     pl->blocks = 0;
     if (pl->mma) {
         const bool shared_mask = pl->mode != MODE_LIST || (d->mask_heads == 1 && !pl->select);
@@ -350,6 +357,41 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
             }
         }
     }
+    // Per-head-list form (list masks per kv or query head, fused selection): the tables every head of a
+    // request shares are built once per block, each head only derives which window candidates it keeps.
+    if (pl->mma && pl->mma_kw == 1 && pl->group_w == 0 && !(p->plan_flags & DSA_PLAN_NO_GROUP) &&
+        pl->mode == MODE_LIST && p->num_kv_heads % kHeadsWarps == 0) {
+        const bool forced = (p->plan_flags & DSA_PLAN_GROUP) != 0;
+        const int64_t lp = p->max_prompt_len > 0 ? p->max_prompt_len : p->max_seq_len;
+        const int64_t dir_cap = std::min<int64_t>(p->max_seq_len, lp + d->n_sink);
+        const int64_t kcap = std::min<int64_t>(d->window, (int64_t)d->n_att * (pl->headmask ? G : 1) + d->n_sink);
+        Plan probe = *pl;
+        probe.heads = true;
+        probe.dir_cap = (int)std::max<int64_t>(dir_cap, 1);
+        probe.kidx_cap = (int)std::max<int64_t>(kcap, 1);
+        KernelShape hs = {};
+        const int32_t rch = dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
+            using T = decltype(t);
+            return kernel_shape<T, decltype(dd)::value>(kernel_query(probe), pl->chunk, pl->bitmap_words, &hs)
+                       ? DSA_OK : DSA_ERR_UNSUPPORTED;
+        });
+        // two blocks per SM or nothing: with one, a block's set-up has nobody to hide behind
+        if (rch == DSA_OK && hs.smem <= 112 * 1024 && d->window <= 65536 && (!forced || (p->plan_flags & DSA_PLAN_GROUP_W4))) {
+            int u = (int)((p->plan_flags & DSA_PLAN_HEADS_PER_WARP_MASK) >> DSA_PLAN_HEADS_PER_WARP_SHIFT);
+            if (!forced || u < 1) {
+                int stages_unused = 0;
+                u = choose_heads_per_warp(p, *pl, kHeadsWarps, bound, hs.smem, 0, kNumSMs, &stages_unused);
+            }
+            if (u >= 1 && p->num_kv_heads % (kHeadsWarps * u) == 0) {
+                pl->heads = true;
+                pl->dir_cap = probe.dir_cap;
+                pl->kidx_cap = probe.kidx_cap;
+                pl->group_u = u;
+                pl->mma_warps = 1;
+                pl->blocks = (int64_t)p->batch * pl->n_split * (p->num_kv_heads / (kHeadsWarps * u));
+            }
+        }
+    }
     rc = shape_of(pl->chunk, &shape);                         // (the small-launch form may have been chosen since)
     if (rc != DSA_OK) return rc;
     pl->stages = shape.stages;
@@ -366,7 +408,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     // loss of 10 % on the dense calls at batch 1-8).
     const bool force_shallow = (p->plan_flags & DSA_PLAN_RING_SHALLOW) != 0;
     const bool force_deep = (p->plan_flags & DSA_PLAN_RING_DEEP) != 0 && !force_shallow;
-    if (pl->mma && pl->group_w == 0 && pl->mma_warps == 2 && pl->mma_kw == 1 && p->split_tokens == 0 &&
+    if (pl->mma && pl->group_w == 0 && !pl->heads && pl->mma_warps == 2 && pl->mma_kw == 1 && p->split_tokens == 0 &&
         (pl->n_split == 1 || force_shallow) && !force_deep) {
         Plan alt = *pl;
         alt.mma_stages = kMmaStagesShallow;
@@ -444,6 +486,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.bitmap_words = pl.bitmap_words;
     a->chunk = pl.chunk; a->n_split = pl.n_split;
     a->heads_per_warp = pl.group_u;
+    a->dir_cap = pl.dir_cap; a->kidx_cap = pl.kidx_cap;
     a->n_items = (int)pl.grid;
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
@@ -618,9 +661,11 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->split_tokens = pl.chunk;
     info->n_split = pl.n_split;
     info->launches = problem->batch == 0 ? 0 : (pl.n_split > 1 ? 2 : 1);
-    info->grid_blocks = (int32_t)(pl.group_w > 0 ? pl.blocks : (pl.mma ? pl.grid / pl.mma_warps : pl.grid));
-    info->heads_per_block = pl.group_w * pl.group_u;
-    info->block_warps = pl.mma ? (pl.group_w > 0 ? pl.group_w : pl.mma_warps * pl.mma_kw) : 4;
+    const int block_warps = pl.heads ? kHeadsWarps : pl.group_w;        // (0: one of the one-block-per-item kernels)
+    info->grid_blocks = (int32_t)(block_warps > 0 ? pl.blocks : (pl.mma ? pl.grid / pl.mma_warps : pl.grid));
+    info->heads_per_block = block_warps * pl.group_u;
+    info->block_warps = pl.mma ? (block_warps > 0 ? block_warps : pl.mma_warps * pl.mma_kw) : 4;
+    info->per_head_lists = pl.heads ? 1 : 0;
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;
     info->tensor_cores = pl.mma ? 1 : 0;

@@ -29,7 +29,9 @@ struct AttnArgs {
     int B, H_q, H_kv;
     float scale_log2;            // sm_scale * log2(e)
     MaskArgs mask;
-    int heads_per_warp;          // head-group kernel: kv heads each warp streams back to back through one row list
+    int heads_per_warp;          // head-group / per-head-list kernels: kv heads each warp streams back to back
+    int dir_cap;                 // per-head-list kernel: capacity of the always-kept-row table (rows)
+    int kidx_cap;                //                       and of a head's kept-candidate list (rows)
     int chunk;                   // kept rows per split (multiple of the tile; see MAX_CHUNK)
     int n_split;
     int n_items;                 // B * H_kv * n_split work items
@@ -115,6 +117,18 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src,
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+// Wait until at most min(n, MAXN) of this thread's cp.async groups are still pending (n >= 0 known
+// only at run time; the instruction takes an immediate).
+template <int MAXN>
+__device__ __forceinline__ void cp_async_wait_upto(int n) {
+    if constexpr (MAXN > 0) {
+        if (n >= MAXN) cp_async_wait<MAXN>();
+        else cp_async_wait_upto<MAXN - 1>(n);
+    } else {
+        cp_async_wait<0>();
+    }
+}
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;

@@ -4,6 +4,7 @@
 #include "dsa_attn.cuh"
 #include "dsa_attn_mma.cuh"
 #include "dsa_attn_group.cuh"
+#include "dsa_attn_heads.cuh"
 #include "dsa_launch.cuh"
 
 #include <atomic>
@@ -116,6 +117,26 @@ struct KernelPick {
         return stages == kGroupStagesShallow ? launch_group_s<kGroupStagesShallow>(w, append, a, blocks, smem_bytes, st)
                                              : launch_group_s<kGroupStages>(w, append, a, blocks, smem_bytes, st);
     }
+    // Per-head-list tensor-core kernel (bf16, list masks per kv or query head, fused selection).
+    static size_t smem_heads(int dir_cap, int window, int kidx_cap, int bw) {
+        return HeadsCfg<D, G, kMmaStages, kHeadsWarps, HM>::smem_bytes(dir_cap, window, kidx_cap, bw);
+    }
+    template <bool APPEND>
+    static ConfiguredFlags* heads_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    template <bool APPEND>
+    static cudaError_t launch_heads_a(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
+        if constexpr (sizeof(T) == 2) {
+            auto kern = dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, APPEND>;
+            const cudaError_t e = ensure_configured(kern, heads_configured<APPEND>());
+            if (e != cudaSuccess) return e;
+            return launch_pdl(kern, (unsigned)blocks, 32 * kHeadsWarps, smem_bytes, st, a);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
+    static cudaError_t launch_heads(bool append, const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
+        return append ? launch_heads_a<true>(a, blocks, smem_bytes, st) : launch_heads_a<false>(a, blocks, smem_bytes, st);
+    }
     // Configure every kernel of this variant for the current device (see dsa_prepare).
     static cudaError_t prepare() {
         cudaError_t e = ensure_configured(dsa_attn_kernel<T, D, G, TILE, STAGES, HM, SEL>, cc_configured());
@@ -127,6 +148,10 @@ struct KernelPick {
                     e = ensure_configured(dsa_attn_mma_kernel<D, G, ST, HM, SEL, W, APPEND, KW>,
                                           mma_configured<W, APPEND, KW, ST>());
             };
+            if (e == cudaSuccess)
+                e = ensure_configured(dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, false>, heads_configured<false>());
+            if (e == cudaSuccess)
+                e = ensure_configured(dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, true>, heads_configured<true>());
             using one = std::integral_constant<int, 1>;
             using two = std::integral_constant<int, 2>;
             using four = std::integral_constant<int, kMmaItemWarps>;
@@ -214,6 +239,11 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
     return dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
         out->tile = q.mma ? MMA_KEYS : P::TILE;
+        if (q.mma && q.heads) {
+            out->stages = kMmaStages;
+            out->smem = P::smem_heads(q.dir_cap, q.window, q.kidx_cap, bitmap_words);
+            return;
+        }
         if (q.mma && q.group_w > 0) {
             out->stages = q.group_stages == kGroupStagesShallow ? kGroupStagesShallow : kGroupStages;
             out->smem = P::smem_group(q.group_w, out->stages, chunk, bitmap_words);
@@ -233,7 +263,8 @@ cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, 
     cudaError_t err = cudaErrorInvalidValue;
     dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
-        if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
+        if (q.mma && q.heads) err = P::launch_heads(append, a, blocks, smem, st);
+        else if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
         else
         err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, q.mma_stages, a, items, smem, st, append)
                     : P::launch(a, items, smem, st);

@@ -10,6 +10,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kMmaItemWarps = 4;                   // warps per work item in small launches
 constexpr int kMmaStages = 3;                      // ring slots per warp: two 16-key tiles in flight, one being consumed
 constexpr int kMmaStagesShallow = 2;
+constexpr int kHeadsWarps = 4;                     // warps per block of the per-head-list kernel
 constexpr int kGroupStagesShallow = 2;             // shallow form: half as many blocks again per SM
 constexpr int kGroupStages = 3;                    // ring slots per warp of the head-group kernel (4 and 6 slots with
                                                    // fewer warps per SM measured 25-45 % slower: the warps, not the
@@ -27,6 +28,8 @@ struct KernelQuery {
     int group_w;             // head-group tensor-core kernel: warps per block that share one row list for
                              // group_w x heads_per_warp kv heads (2 or 4); 0: not that kernel
     int group_stages;        // its ring depth: kGroupStages or kGroupStagesShallow
+    bool heads;              // per-head-list tensor-core kernel (blocks of kHeadsWarps warps); sizes of its tables:
+    int dir_cap, kidx_cap, window;
 };
 
 struct KernelShape {

@@ -1,12 +1,15 @@
-"""The head-group form of the tensor-core kernel: one row list per (request, split), built by a
-block of W warps, every warp streaming U kv heads through it back to back.
+"""The multi-head forms of the tensor-core kernel: blocks of W warps, every warp streaming U kv heads
+back to back through one ring.  With a mask that does not depend on the head the block builds ONE
+row list for all of them (head-group kernel); with per-head list masks and the fused selection it
+builds the tables the heads share and every head derives its own list of kept window candidates
+(per-head-list kernel, 4 warps per block).
 
-The planner takes it by itself only where it measured faster; here it is forced, in several
-(W, U) shapes, onto the cases of the other GPU test modules -- the five configurations, the small
-shapes with and without splits, degenerate requests, poisoned skipped rows, the fused decode step
-and its loops, bounded ring caches, the randomised problems -- so that what those modules pin to
-the oracle is pinned for this kernel too.  (Calls it cannot serve -- per-head masks, the fused
-selection, float32, head counts that W x U does not divide -- run on the other kernels as before.)"""
+The planner chooses W, U and the ring depth by itself; here several (W, U) shapes are forced onto
+the cases of the other GPU test modules -- the five configurations, the small shapes with and
+without splits, degenerate requests, poisoned skipped rows, the fused decode step and its loops,
+the phase-2 selection, bounded ring caches, the randomised problems -- so that what those modules
+pin to the oracle is pinned for every shape of these kernels.  (Calls they cannot serve -- float32,
+head counts that W x U does not divide -- run on the other kernels as before.)"""
 import pytest
 import torch
 
@@ -15,6 +18,7 @@ from tests import test_gpu_decode_step as t_step
 from tests import test_gpu_fuzz as t_fuzz
 from tests import test_gpu_parity as t_parity
 from tests import test_gpu_ring_append as t_ring
+from tests import test_gpu_selection as t_sel
 
 pytestmark = pytest.mark.gpu
 
@@ -58,12 +62,19 @@ def test_the_switch_really_selects_the_head_group_kernel(dsa, forced):
                 assert plan.grid_blocks * w_ * u_ == plan.work_items and plan.item_warps == 1
             else:
                 assert plan.heads_per_block == 0
-        # one mask per query head: the switch is ignored
+        # one mask per query head, with and without the fused selection: the per-head-list kernel (4 warps)
         per_head = synth.random_valid_trace(__import__("numpy").random.default_rng(0), w.window, w.n_att,
                                             (w.batch, w.num_q_heads))
-        if w.num_q_heads > 1:
-            diag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=torch.from_numpy(per_head).cuda())
-            assert dsa.dsa_query_plan(prob, diag).heads_per_block == 0
+        for select in (False, True):
+            diag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=torch.from_numpy(per_head).cuda(),
+                            select=select)
+            plan = dsa.dsa_query_plan(prob, diag)
+            if w_ == 4 and w.num_kv_heads % (4 * u_) == 0 and w.index != 4:
+                assert plan.per_head_lists == 1 and plan.heads_per_block == 4 * u_ and plan.block_warps == 4
+            elif w.index != 4:
+                assert plan.per_head_lists == 0
+            # (window 1024 with four masks per kv head: the per-head tables leave no room for two blocks
+            # per SM, so that configuration stays with the one-warp-per-item kernel)
     # float32 has no tensor-core path: the switch is ignored
     w = synth.workload(1)
     prob = dsa.problem_from_host(synth.make_inputs(w), dtype=torch.float32)
@@ -89,7 +100,7 @@ def test_splits_degenerate_requests_and_poisoned_rows(dsa, forced):
     t_parity.test_skipped_rows_are_never_read(dsa)
 
 
-@pytest.mark.parametrize("mask", ["dense", "grid_sink", "window", "list_heads"])
+@pytest.mark.parametrize("mask", ["dense", "grid_sink", "window", "list_heads", "list_select"])
 @pytest.mark.parametrize("name", sorted(t_step.WORKLOADS))
 def test_fused_decode_step(dsa, forced, name, mask):
     for split in (0, 48):
@@ -100,6 +111,13 @@ def test_fused_decode_step_full_request_and_loops(dsa, forced):
     t_step.test_a_full_request_drops_its_token(dsa)
     for use_graph in (False, True):
         t_step.test_fused_decode_loop_two_layers_one_seq_len(dsa, use_graph)
+
+
+def test_phase2_selection(dsa, forced):
+    params = [mk.args[1] for mk in t_sel.test_every_step_of_one_sequence.pytestmark if mk.name == "parametrize"][0]
+    for hq, hkv, d, split, n_sink, positional in params:
+        t_sel.test_every_step_of_one_sequence(dsa, hq, hkv, d, split, n_sink, positional)
+    t_sel.test_free_running_decode_loop_grows_a_valid_trace(dsa)
 
 
 def test_bounded_ring_caches(dsa, forced):
