@@ -133,6 +133,9 @@ typedef struct dsa_problem {
 #define DSA_PLAN_GROUP         0x10u  /* take the head-group / per-head-list kernels wherever they can run */
 #define DSA_PLAN_NO_GROUP      0x20u  /* never take them                                                 */
 #define DSA_PLAN_GROUP_W4      0x40u  /* forced head-group kernel: 4 warps per block instead of 2        */
+#define DSA_PLAN_NO_CLUSTER    0x80u  /* small launches: never let a thread-block cluster share a work item */
+#define DSA_PLAN_CLUSTER2      0x10000u /* small launches (several warps per item): clusters of 2 blocks  */
+#define DSA_PLAN_CLUSTER4      0x20000u /*                                           clusters of 4 blocks  */
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u
 
@@ -208,6 +211,8 @@ typedef struct dsa_plan_info {
     int32_t block_warps;    /* warps per thread block                                              */
     int32_t per_head_lists; /* 1: the per-head-list tensor-core kernel (list masks per head, fused  */
                             /* selection): shared tables per block, one candidate list per head    */
+    int32_t cluster_blocks; /* blocks of a thread-block cluster that share one work item and merge */
+                            /* through distributed shared memory (small launches); 1: no cluster   */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);

@@ -23,6 +23,7 @@ DSA_MASK_WINDOW, DSA_MASK_GRID, DSA_MASK_LIST = 0, 1, 2
 DSA_PLAN_CUDA_CORES, DSA_PLAN_NO_ITEM_WARPS, DSA_PLAN_RING_DEEP, DSA_PLAN_RING_SHALLOW = 0x1, 0x2, 0x4, 0x8
 DSA_PLAN_GROUP, DSA_PLAN_NO_GROUP, DSA_PLAN_GROUP_W4 = 0x10, 0x20, 0x40
 DSA_PLAN_HEADS_PER_WARP_SHIFT = 8
+DSA_PLAN_NO_CLUSTER, DSA_PLAN_CLUSTER2, DSA_PLAN_CLUSTER4 = 0x80, 0x10000, 0x20000
 
 
 def plan_group(warps: int, heads_per_warp: int) -> int:
@@ -68,7 +69,8 @@ class dsa_plan_info(ctypes.Structure):
                 ("smem_bytes", ctypes.c_int32), ("tile_tokens", ctypes.c_int32),
                 ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32),
                 ("item_warps", ctypes.c_int32), ("heads_per_block", ctypes.c_int32),
-                ("block_warps", ctypes.c_int32), ("per_head_lists", ctypes.c_int32)]
+                ("block_warps", ctypes.c_int32), ("per_head_lists", ctypes.c_int32),
+                ("cluster_blocks", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:

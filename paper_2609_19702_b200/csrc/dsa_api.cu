@@ -44,7 +44,8 @@ int sm_count() {
 
 constexpr uint32_t kKnownPlanFlags = DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_RING_DEEP |
                                      DSA_PLAN_RING_SHALLOW | DSA_PLAN_GROUP | DSA_PLAN_NO_GROUP |
-                                     DSA_PLAN_GROUP_W4 | DSA_PLAN_HEADS_PER_WARP_MASK;
+                                     DSA_PLAN_GROUP_W4 | DSA_PLAN_HEADS_PER_WARP_MASK | DSA_PLAN_NO_CLUSTER |
+                                     DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -63,6 +64,7 @@ struct Plan {
     bool mma;            // bf16: one warp per work item, tensor-core tiles
     int mma_warps;       // warps (= kv heads) per block that share one row list
     int mma_kw;          // warps that share one work item (small launches), 1 or kMmaItemWarps
+    int mma_cl;          // and blocks of a thread-block cluster that share it (1: no cluster)
     int mma_stages;      // ring depth of the tensor-core kernel
     int group_w;         // head-group tensor-core kernel: warps per block (0: not that kernel)
     int group_u;         // and kv heads each warp streams through the block's one row list
@@ -93,6 +95,7 @@ KernelQuery kernel_query(const Plan& pl) {
     KernelQuery q;
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
     q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
+    q.mma_cl = pl.mma_cl;
     q.group_w = pl.group_w; q.group_stages = pl.group_stages;
     q.heads = pl.heads; q.dir_cap = pl.dir_cap; q.kidx_cap = pl.kidx_cap; q.window = pl.window;
     return q;
@@ -242,6 +245,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->mma = p->dtype == DSA_BF16 && !(p->plan_flags & DSA_PLAN_CUDA_CORES);
     pl->mma_warps = 1;
     pl->mma_kw = 1;
+    pl->mma_cl = 1;
     pl->mma_stages = kMmaStages;
     pl->group_w = 0;
     pl->group_u = 0;
@@ -295,10 +299,13 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
         // single launch still wins there).  Requests beyond 2048 rows need the combine anyway;
         // there the merge on top of it measured as a small loss.
         // (a forced head-group kernel takes the place of the small-launch form as well)
-        if (pl->mma && want_split >= 2 && bound <= 2 * MAX_CHUNK &&
+        // (a forced cluster size brings this form with it: clusters exist only on top of it)
+        const bool cluster_forced = (p->plan_flags & (DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4)) != 0 &&
+                                    !pl->headmask && !pl->select;
+        if (pl->mma && (want_split >= 2 || cluster_forced) && bound <= 2 * MAX_CHUNK &&
             !(p->plan_flags & (DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_GROUP))) {
             const int64_t kw_blocks = pairs * ((want_split + kMmaItemWarps - 1) / kMmaItemWarps);
-            if (kw_blocks <= 2 * kNumSMs || kw_blocks >= 4 * kNumSMs || bound > MAX_CHUNK) {
+            if (cluster_forced || kw_blocks <= 2 * kNumSMs || kw_blocks >= 4 * kNumSMs || bound > MAX_CHUNK) {
                 pl->mma_kw = kMmaItemWarps;
                 pl->mma_warps = 1;
                 want_split = (want_split + kMmaItemWarps - 1) / kMmaItemWarps;
@@ -306,6 +313,26 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
             }
         }
         want_split = std::max<int64_t>(want_split, (bound + max_chunk - 1) / max_chunk);
+        // Smaller launches still: a CLUSTER of 2 or 4 such blocks shares the item (8 or 16 warps with one
+        // to three tiles each, all in flight at once) and block 0 collects the others' states through
+        // distributed shared memory -- while every block of every cluster is resident at once (two
+        // blocks per SM) and a block still gets a few tiles.  Head-independent masks, no HBM splits.
+        // (Measured, single calls with a cold L2: GQA long-sequence configuration 18.4 -> 16.4 us, paged
+        // workload at batch 1 / 2: 16.4 -> 14.3 us with clusters of four; clusters of two at batch 4: no
+        // change; clusters that do not all fit at once lose: batch 8, 22.5 -> 26.7 / 38.9 us.)
+        // Where the plan would otherwise cut the item into 2-4 splits with partials in HBM and a combine
+        // launch, the cluster takes the place of those splits.
+        int cluster = 1;
+        if (pl->mma_kw > 1 && want_split <= 4 && !pl->headmask && !pl->select && !(p->plan_flags & DSA_PLAN_NO_CLUSTER)) {
+            const int forced = (p->plan_flags & DSA_PLAN_CLUSTER4) ? 4 : ((p->plan_flags & DSA_PLAN_CLUSTER2) ? 2 : 0);
+            if (forced) cluster = forced >= want_split ? forced : 1;
+            else if (pairs * 4 <= 2 * kNumSMs && bound >= 4 * 96) cluster = 4;
+            else if (want_split <= 2 && pairs * 2 <= 2 * kNumSMs && bound >= 2 * 96) cluster = 2;
+        }
+        if (cluster > 1) {
+            pl->mma_cl = cluster;
+            want_split = cluster;                             // (row ranges per block; the result is final: n_split is reset below)
+        }
         // Requests too long for one row list are split anyway; when the (request, kv head) pairs
         // alone fill half the device's warp slots, ~512-row items balance better across the SMs
         // than ~900-row ones (measured on dense calls: +3-10 % at 640-4096 pairs, a loss below).
@@ -316,6 +343,11 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     }
     pl->chunk = chunk;
     pl->n_split = (int)((bound + chunk - 1) / chunk);
+    if (pl->mma_cl > 1) {
+        // the blocks of a cluster cover the row ranges [r chunk, (r + 1) chunk) and merge on chip
+        if (pl->n_split > pl->mma_cl || p->split_tokens > 0) pl->mma_cl = 1;
+        else pl->n_split = 1;
+    }
     if (pl->n_split > kMaxSplits) return DSA_ERR_UNSUPPORTED;   // the combine kernel holds one weight per split
     pl->grid = (int64_t)p->batch * p->num_kv_heads * pl->n_split;
     if (pl->grid > 0x7fffffffLL) return DSA_ERR_UNSUPPORTED;
@@ -666,6 +698,8 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->heads_per_block = block_warps * pl.group_u;
     info->block_warps = pl.mma ? (block_warps > 0 ? block_warps : pl.mma_warps * pl.mma_kw) : 4;
     info->per_head_lists = pl.heads ? 1 : 0;
+    info->cluster_blocks = pl.mma_cl;
+    if (pl.mma_cl > 1) info->grid_blocks = (int32_t)(pl.grid * pl.mma_cl);
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;
     info->tensor_cores = pl.mma ? 1 : 0;

@@ -55,6 +55,25 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
+// ---- thread-block clusters: the CTAs of a cluster share one work item (see CL below) -------------
+__device__ __forceinline__ unsigned cluster_ctarank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// split cluster barrier: every thread of every CTA arrives, and waits where it needs the others
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// a float of CTA `rank`'s shared memory, at the place where this CTA has `local` (distributed shared memory)
+__device__ __forceinline__ float ld_cluster_f32(const float* local, unsigned rank) {
+    unsigned remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                 : "=r"(remote) : "r"((unsigned)__cvta_generic_to_shared(local)), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
 template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W = 1>
 struct MmaCfg {
     using T = __nv_bfloat16;
@@ -92,7 +111,14 @@ struct MmaItemCfg {
 // warps share one work item instead of the item being cut into KW splits with a combine launch
 // behind them: they build the row list together, warp k streams tiles k, k + KW, ... through its
 // own ring, and the partial softmax states are merged through shared memory at the end.
-template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false, int KW = 1>
+//
+// CL > 1: smaller launches still.  A thread-block CLUSTER of CL such blocks shares the work item:
+// block r of the cluster builds and streams rows [r chunk, (r + 1) chunk) of the kept sequence (so
+// CL x KW warps have one to three tiles each, all in flight at once), merges its warps as above, and
+// block 0 then reads the other blocks' merged states straight out of their shared memory
+// (ld.shared::cluster after a cluster barrier) and writes the result: no partials in HBM, no combine
+// launch.  The launch carries the cluster dimension; plain per-thread loads only cross the cluster.
+template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false, int KW = 1, int CL = 1>
 __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArgs a) {
     using C = MmaCfg<D, G, STAGES, HEADMASK, SELECT, W * KW>;   // one ring per warp
     using IC = MmaItemCfg<D, G, HEADMASK, SELECT>;
@@ -101,6 +127,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     constexpr int NW = W * KW;                            // warps per block
     static_assert(W == 1 || (!HEADMASK && !SELECT), "a shared row list needs a head-independent mask");
     static_assert(W == 1 || KW == 1, "several warps per head only with one head per block");
+    static_assert(CL == 1 || (KW > 1 && !SELECT), "clusters extend the several-warps-per-item form");
 
     // Programmatic launch on both sides: a combine kernel queued behind this grid may be scheduled
     // from now on (it waits for this grid to finish before it reads anything), and this grid may
@@ -120,9 +147,12 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     // kv heads vary fastest across the grid: the warps that run together read the same tokens
     // of neighbouring heads, i.e. neighbouring memory.
     const int hblocks = a.H_kv / W;
-    const int kvh = (blockIdx.x % hblocks) * W + hw;
-    const int split = (blockIdx.x / hblocks) % a.n_split;
-    const int b = blockIdx.x / (hblocks * a.n_split);
+    // (cluster form: the CL blocks of a cluster are consecutive and take the "splits" of one pair;
+    // a.n_split is 1 there, the result is final)
+    const int item_block = CL > 1 ? blockIdx.x / CL : blockIdx.x;
+    const int kvh = (item_block % hblocks) * W + hw;
+    const int split = CL > 1 ? (int)cluster_ctarank() : (item_block / hblocks) % a.n_split;
+    const int b = CL > 1 ? item_block / hblocks : item_block / (hblocks * a.n_split);
 
     const int seq_raw = a.seq_len[b], prompt_raw = req_prompt_len(a, b);
     // ---- Q^T as B operand: head = lane / 4, dims 2*(lane%4)+{0,1} (+8) of every 16-dim step ----
@@ -212,13 +242,14 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
         const int c = lane < C::CPR ? lane : lane - C::CPR;
         *reinterpret_cast<uint4*>(base + (off_new + (int64_t)kvh * a.stride_head) * 2 + c * 16) = new_chunk;
     }
-    if (n_rows <= 0) {
+    if (CL == 1 && n_rows <= 0) {
         if (wk == 0) write_empty_item<IC, 32>(a, m, b, kvh, split, lane);
         return;
     }
+    // (a block of a cluster that got no rows goes on with zero tiles: the others wait for it)
     sync_builders();                                   // the last barrier: from here on warps run free
     // kept positions ascend, so the token being decoded can only be this item's last row
-    if (APPEND && has_new && list.rowoff[n_rows - 1] == off_new + (int64_t)list_kvh * a.stride_head)
+    if (APPEND && has_new && n_rows > 0 && list.rowoff[n_rows - 1] == off_new + (int64_t)list_kvh * a.stride_head)
         new_r = n_rows - 1;
     const int item_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
     const int n_tiles = item_tiles > wk ? (item_tiles - wk + KW - 1) / KW : 0;      // this warp's
@@ -353,7 +384,8 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
             }
         }
         __syncthreads();
-        if (wk > 0) return;
+        if (CL == 1 && wk > 0) return;
+        if (wk == 0)
         for (int w = 1; w < KW; ++w) {
             const float* other = rec + (size_t)(w - 1) * REC * 32 + lane;
 #pragma unroll
@@ -376,6 +408,52 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
                     if (ov < bv[j] || (ov == bv[j] && op < bp[j])) { bv[j] = ov; bp[j] = op; }
                 }
             }
+        }
+    }
+    if (CL > 1) {
+        // Merge across the cluster.  Every thread of every block passes the same two barriers:
+        //   blocks 1.. leave their merged state in their OWN shared memory   -> barrier 1 ->
+        //   block 0 reads it there (distributed shared memory) and folds it in -> barrier 2 ->
+        //   the other blocks may exit (their memory is no longer needed).
+        constexpr int REC = C::MTILES * 4 + 8;
+        float* rec = reinterpret_cast<float*>(smem) + lane;       // (warp 0 is done with the other warps' records)
+        if (wk == 0 && split > 0) {
+#pragma unroll
+            for (int mt = 0; mt < C::MTILES; ++mt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) rec[(mt * 4 + e) * 32] = o[mt][e];
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                rec[(C::MTILES * 4 + j) * 32] = mrun[j];
+                rec[(C::MTILES * 4 + 2 + j) * 32] = ltot[j];
+            }
+        }
+        cluster_arrive();
+        cluster_wait();
+        if (wk == 0 && split == 0) {
+            for (unsigned r = 1; r < (unsigned)CL; ++r) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const float m_o = ld_cluster_f32(rec + (C::MTILES * 4 + j) * 32, r);
+                    const float l_o = ld_cluster_f32(rec + (C::MTILES * 4 + 2 + j) * 32, r);
+                    const float mnew = fmaxf(mrun[j], m_o);
+                    const float msafe = mnew == -INFINITY ? 0.f : mnew;
+                    const float c0 = fast_exp2(mrun[j] - msafe), c1 = fast_exp2(m_o - msafe);
+                    ltot[j] = ltot[j] * c0 + l_o * c1;
+                    mrun[j] = mnew;
+#pragma unroll
+                    for (int mt = 0; mt < C::MTILES; ++mt) {
+                        o[mt][j] = o[mt][j] * c0 + ld_cluster_f32(rec + (mt * 4 + j) * 32, r) * c1;
+                        o[mt][2 + j] = o[mt][2 + j] * c0 + ld_cluster_f32(rec + (mt * 4 + 2 + j) * 32, r) * c1;
+                    }
+                }
+            }
+        }
+        cluster_arrive();
+        if (wk > 0 || split > 0) {
+            cluster_wait();
+            return;
         }
     }
 #pragma unroll
@@ -415,6 +493,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
             }
         }
     }
+    if (CL > 1) cluster_wait();                           // (barrier 2, for form's sake: every arrival is waited for)
 }
 
 }  // namespace dsa

@@ -31,6 +31,27 @@ cudaError_t launch_pdl(Kern kern, unsigned grid, unsigned block, size_t smem, cu
     return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
+// The same with a thread-block cluster of `cluster` blocks along x (grid must be a multiple of it).
+template <class Kern, class... Args>
+cudaError_t launch_pdl_cluster(Kern kern, unsigned grid, unsigned block, size_t smem, cudaStream_t st, unsigned cluster,
+                               Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 template <typename T, int D, int G, bool HM, bool SEL>
 struct KernelPick {
     // Small tiles (2 KB of K + 2 KB of V) in a 4-deep ring: 16-20 KB of shared memory per block, so
@@ -73,6 +94,25 @@ struct KernelPick {
     }
     template <int W, bool APPEND, int KW, int ST>
     static ConfiguredFlags* mma_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    template <bool APPEND, int CL>
+    static ConfiguredFlags* cluster_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    // several warps per item, CL blocks of a cluster per item (head-independent masks only)
+    template <bool APPEND, int CL>
+    static cudaError_t launch_cluster_c(const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
+        if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, CL>;
+            const cudaError_t e = ensure_configured(kern, cluster_configured<APPEND, CL>());
+            if (e != cudaSuccess) return e;
+            return launch_pdl_cluster(kern, (unsigned)(items * CL), 32 * kMmaItemWarps, smem_bytes, st, CL, a);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
+    static cudaError_t launch_cluster(int cl, bool append, const AttnArgs& a, int64_t items, size_t smem_bytes,
+                                      cudaStream_t st) {
+        if (cl == 4) return append ? launch_cluster_c<true, 4>(a, items, smem_bytes, st) : launch_cluster_c<false, 4>(a, items, smem_bytes, st);
+        return append ? launch_cluster_c<true, 2>(a, items, smem_bytes, st) : launch_cluster_c<false, 2>(a, items, smem_bytes, st);
+    }
     static ConfiguredFlags* cc_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
 
     template <int W, bool APPEND, int KW, int ST = kMmaStages>
@@ -162,6 +202,17 @@ struct KernelPick {
             mma(one{}, std::false_type{}, four{}, deep{});
             mma(one{}, std::true_type{}, four{}, deep{});
             if constexpr (!HM && !SEL) {
+                auto cluster = [&](auto app, auto cl) {
+                    constexpr bool APPEND = decltype(app)::value;
+                    constexpr int CL = decltype(cl)::value;
+                    if (e == cudaSuccess)
+                        e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, CL>,
+                                              cluster_configured<APPEND, CL>());
+                };
+                cluster(std::false_type{}, two{});
+                cluster(std::true_type{}, two{});
+                cluster(std::false_type{}, four{});
+                cluster(std::true_type{}, four{});
                 auto group = [&](auto w, auto app, auto stg) {
                     constexpr int W = decltype(w)::value, ST = decltype(stg)::value;
                     constexpr bool APPEND = decltype(app)::value;
@@ -263,7 +314,8 @@ cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, 
     cudaError_t err = cudaErrorInvalidValue;
     dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
-        if (q.mma && q.heads) err = P::launch_heads(append, a, blocks, smem, st);
+        if (q.mma && q.mma_kw > 1 && q.mma_cl > 1) err = P::launch_cluster(q.mma_cl, append, a, items, smem, st);
+        else if (q.mma && q.heads) err = P::launch_heads(append, a, blocks, smem, st);
         else if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
         else
         err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, q.mma_stages, a, items, smem, st, append)

@@ -24,6 +24,7 @@ struct KernelQuery {
     bool mma;                // tensor-core kernel (bf16) rather than the CUDA-core kernel
     int mma_warps;           // tensor-core kernel: kv heads per block that share one row list (1 or 2)
     int mma_kw;              // tensor-core kernel: warps that share one work item (1 or kMmaItemWarps)
+    int mma_cl;              // tensor-core kernel, several warps per item: blocks of a cluster that share the item (1, 2 or 4)
     int mma_stages;          // tensor-core kernel: kMmaStages, or kMmaStagesShallow (two heads per block only)
     int group_w;             // head-group tensor-core kernel: warps per block that share one row list for
                              // group_w x heads_per_warp kv heads (2 or 4); 0: not that kernel

@@ -134,7 +134,12 @@ def test_small_launch_plan_shares_items_between_warps(dsa):
     # 8 requests x 8 kv heads cannot fill the device: four warps per item, no split, one launch
     rc, info = _plan(dsa, _problem(dsa, batch=8), _diag(dsa))
     assert rc == 0 and info.tensor_cores == 1 and info.item_warps == 4
-    assert info.n_split == 1 and info.launches == 1 and info.split_tokens >= 64 + 410
+    # ... and a cluster of four such blocks per item (64 x 4 blocks fit the device at once), each block a
+    # quarter of the rows; still one launch and no partial results
+    assert info.n_split == 1 and info.launches == 1 and info.cluster_blocks == 4
+    assert info.split_tokens * info.cluster_blocks >= 64 + 410 and info.grid_blocks == 64 * 4
+    rc, info = _plan(dsa, _problem(dsa, batch=8, plan_flags=dsa.DSA_PLAN_NO_CLUSTER), _diag(dsa))
+    assert rc == 0 and info.item_warps == 4 and info.cluster_blocks == 1 and info.split_tokens >= 64 + 410
     # the same requests without a mask are longer than one row list: split, one warp per item
     rc, info = _plan(dsa, _problem(dsa, batch=8))
     assert rc == 0 and info.item_warps == 1 and info.n_split > 1 and info.launches == 2

@@ -79,7 +79,8 @@ def test_shared_item_path_agrees_with_one_warp_per_item(dsa, name, make, splits)
             if diag is not None:
                 assert plan.item_warps == (4 if setting == "1" else 1), name
                 if setting == "1":
-                    assert plan.n_split == splits, name
+                    # (a cluster of blocks takes the place of HBM splits where the mask allows one)
+                    assert plan.n_split == (1 if plan.cluster_blocks > 1 else splits), name
             out, lse = dsa.alloc_outputs(prob)
             ws = dsa.alloc_workspace(prob, diag)
             if diag is None:
@@ -116,3 +117,66 @@ def test_shallow_ring_form_matches_the_oracle(dsa):
             assert dsa.dsa_query_plan(prob, g2).stages == 2
         _check_all_modes(dsa, inp2, list_heads=(1,), seed=6, what="shallow ring, forced",
                          plan_flags=dsa.DSA_PLAN_RING_SHALLOW)
+
+
+# ---------------------------------------------------------------- clusters: several blocks per work item
+
+@pytest.mark.parametrize("name,make", [
+    ("config4 GQA, batch 3", lambda: synth.workload(4, batch=3)),
+    ("config5 paged, batch 1", lambda: synth.workload(5, batch=1)),
+    ("config5 paged, window 1024, batch 2 (in place of two splits)", lambda: synth.workload(5, batch=2, window=1024, n_att=416)),
+    ("config3 long prompt, batch 1", lambda: synth.workload(3, batch=1)),
+])
+def test_cluster_form_is_chosen_for_the_smallest_launches_and_matches_the_oracle(dsa, name, make):
+    """The blocks of a thread-block cluster take row ranges of one work item and block 0 collects
+    their softmax states through distributed shared memory: same results as every other plan."""
+    w = make()
+    inp = synth.make_inputs(w)
+    grid = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    plan = _plan(dsa, inp, grid)
+    assert plan.cluster_blocks in (2, 4) and plan.item_warps == 4 and plan.n_split == 1 and plan.launches == 1, name
+    assert plan.grid_blocks == plan.work_items * plan.cluster_blocks
+    _check_all_modes(dsa, inp, list_heads=(1,), seed=11, what=name)
+    # and switched off: the plan without clusters, same results within the summation-order difference
+    prob_on = dsa.problem_from_host(inp)
+    prob_off = dsa.problem_from_host(inp, plan_flags=dsa.DSA_PLAN_NO_CLUSTER)
+    assert dsa.dsa_query_plan(prob_off, grid).cluster_blocks == 1
+    res = []
+    for prob in (prob_on, prob_off):
+        out, lse = dsa.alloc_outputs(prob)
+        dsa.dsa_decode_attention_sparse(prob, grid, out, lse, dsa.alloc_workspace(prob, grid))
+        torch.cuda.synchronize()
+        res.append((out.float().cpu(), lse.cpu()))
+    assert torch.allclose(res[0][0], res[1][0], atol=2e-2, rtol=2e-2) and torch.allclose(res[0][1], res[1][1], atol=1e-4, rtol=0)
+
+
+@pytest.mark.parametrize("flag", ["DSA_PLAN_CLUSTER2", "DSA_PLAN_CLUSTER4"])
+def test_forced_cluster_sizes_on_short_ragged_and_empty_ranges(dsa, flag):
+    """Forced onto requests so short that some blocks of a cluster (and some warps of a block) get no
+    rows at all, with and without the fused decode step."""
+    from tests import test_gpu_decode_step as t_step
+    flags = getattr(dsa, flag)
+    w = synth.Workload("clshort", 93, 6, 8, 2, 128, 3, 20, 15, 0, 300, 80, 1, 300)
+    inp = synth.make_inputs(w, poison=False)
+    inp["position"][:4] = np.array([1, 7, 20, 33])
+    inp["seq_len"][:4] = inp["prompt_len"][:4] + inp["position"][:4]
+    grid = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    prob = dsa.problem_from_host(inp, plan_flags=flags)
+    plan = dsa.dsa_query_plan(prob, grid)
+    assert plan.cluster_blocks == (2 if flag.endswith("2") else 4) and plan.item_warps == 4
+    _check_all_modes(dsa, inp, list_heads=(1,), seed=12, what=flag, plan_flags=flags)
+    # the fused decode step through the same plans
+    orig = dsa.Problem.c_struct
+
+    def patched(self):
+        p = orig(self)
+        p.plan_flags |= flags
+        return p
+
+    dsa.Problem.c_struct = patched
+    try:
+        for name in ("gqa_long", "paged", "gqa8_paged_small"):
+            for mask in ("dense", "grid_sink", "window"):
+                t_step.test_fused_step_matches_oracle_and_the_two_calls(dsa, name, mask, 0)
+    finally:
+        dsa.Problem.c_struct = orig
