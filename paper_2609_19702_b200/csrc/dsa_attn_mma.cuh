@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     const int hblocks = a.H_kv / W;
     // (cluster form: the CL blocks of a cluster are consecutive and take the "splits" of one pair;
     // a.n_split is 1 there, the result is final)
-    const int item_block = CL > 1 ? blockIdx.x / CL : blockIdx.x;
+    const unsigned item_block = CL > 1 ? blockIdx.x / CL : blockIdx.x;
     const int kvh = (item_block % hblocks) * W + hw;
     const int split = CL > 1 ? (int)cluster_ctarank() : (item_block / hblocks) % a.n_split;
     const int b = CL > 1 ? item_block / hblocks : item_block / (hblocks * a.n_split);
@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     // (a block of a cluster that got no rows goes on with zero tiles: the others wait for it)
     sync_builders();                                   // the last barrier: from here on warps run free
     // kept positions ascend, so the token being decoded can only be this item's last row
-    if (APPEND && has_new && n_rows > 0 && list.rowoff[n_rows - 1] == off_new + (int64_t)list_kvh * a.stride_head)
+    if (APPEND && has_new && (CL == 1 || n_rows > 0) && list.rowoff[n_rows - 1] == off_new + (int64_t)list_kvh * a.stride_head)
         new_r = n_rows - 1;
     const int item_tiles = (n_rows + MMA_KEYS - 1) / MMA_KEYS;
     const int n_tiles = item_tiles > wk ? (item_tiles - wk + KW - 1) / KW : 0;      // this warp's
@@ -384,9 +384,8 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
             }
         }
         __syncthreads();
-        if (CL == 1 && wk > 0) return;
-        if (wk == 0)
-        for (int w = 1; w < KW; ++w) {
+        if (CL == 1) { if (wk > 0) return; }
+        for (int w = 1; w < (CL == 1 || wk == 0 ? KW : 1); ++w) {
             const float* other = rec + (size_t)(w - 1) * REC * 32 + lane;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
