@@ -39,10 +39,10 @@ L2_BYTES = 126 << 20
 # DRAM bytes per launch of the timed kernel (dram__bytes_read.sum + dram__bytes_write.sum of an ncu
 # capture), keyed by the workload string of the JSON line; None until a capture of that launch exists.
 NCU_TRAFFIC_BYTES = {
-    # measured with ncu at batch 32: 209.39 MB read + 3.81 MB written per launch; traffic grows in
-    # proportion to the batch, so a batch-256 launch moves 8 x that
+    # measured with ncu at batch 32 (head-group kernel): 209.39 MB read + 4.44 MB written per launch;
+    # traffic grows in proportion to the batch, so a batch-256 launch moves 8 x that
     "config5_paged_sweep B=256 Hq=32 Hkv=32 D=128 Lp=200 grid=64x64+1 paged16 sparse grid-mask window=512 n_att=208":
-        8 * 213_193_600,
+        8 * 213_825_024,
 }
 
 
@@ -58,9 +58,14 @@ def parse_args():
     ap.add_argument("--n-att", type=int, default=None)
     ap.add_argument("--mode", default="sparse", choices=["sparse", "dense"])
     ap.add_argument("--split-tokens", type=int, default=0)
+    ap.add_argument("--plan-flags", type=lambda x: int(x, 0), default=0,
+                    help="dsa_problem.plan_flags for comparison runs (DSA_PLAN_* bits of dsa.h; 0: the library plans)")
     ap.add_argument("--no-variants", action="store_true", help="skip the dense / other-window timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-decode-loop", action="store_true",
+                    help="skip the whole-image decode loop at batch 128 (the paper's shape: 50 prompt tokens, 1024 "
+                         "image tokens, N_att 52)")
     ap.add_argument("--no-per-config", action="store_true",
                     help="skip the table of every configuration (dense and sparse, L2 flushed between calls)")
     ap.add_argument("--all-configs", action="store_true",
@@ -77,6 +82,17 @@ def workload_name(w, mode):
     else:
         s += " dense"
     return s
+
+
+def kernel_name(plan):
+    """Which attention kernel a plan launches (see dsa_plan_info)."""
+    if not plan.tensor_cores:
+        return "dsa_attn_kernel"
+    if plan.per_head_lists:
+        return "dsa_attn_heads_kernel"
+    if plan.heads_per_block:
+        return "dsa_attn_group_kernel"
+    return "dsa_attn_mma_kernel"
 
 
 def measured_peak():
@@ -306,7 +322,9 @@ def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
                          "queries_per_sec": round(w.batch / t_dense, 1),
                          "bytes": b_dense, "GBs": round(b_dense / t_dense / 1e9, 1),
                          "frac_of_peak": round(b_dense / t_dense / 1e9 / peak, 4),
-                         "n_split": plan.n_split, "launches": plan.launches},
+                         "n_split": plan.n_split, "launches": plan.launches, "kernel": kernel_name(plan),
+                         "heads_per_block": plan.heads_per_block, "item_warps": plan.item_warps,
+                         "cluster_blocks": plan.cluster_blocks},
                "sparse": []}
         for window, n_att in (windows or [(w.window, w.n_att)]):
             ww = synth.workload(w.index, batch=w.batch, window=window, n_att=n_att)
@@ -322,7 +340,9 @@ def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
                                   "frac_of_peak": round(b_sp / t_sp / 1e9 / peak, 4),
                                   "speedup_over_dense": round(t_dense / t_sp, 3),
                                   "ideal_byte_ratio": round(b_dense / b_sp, 3),
-                                  "n_split": plan2.n_split, "launches": plan2.launches})
+                                  "n_split": plan2.n_split, "launches": plan2.launches,
+                                  "kernel": kernel_name(plan2), "heads_per_block": plan2.heads_per_block,
+                                  "item_warps": plan2.item_warps, "cluster_blocks": plan2.cluster_blocks})
         rows.append(row)
         del inputs, prob, out, lse, ws
         torch.cuda.empty_cache()
@@ -532,7 +552,7 @@ def run_ours(args):
             max_seq_len=inputs["max_seq_len"], max_prompt_len=w.prompt_len,
             block_table=inputs["block_table"], block_size=inputs["block_size"],
             num_blocks=0 if inputs["block_table"] is None else inputs["block_table"].numel(),
-            split_tokens=split_tokens)
+            split_tokens=split_tokens, plan_flags=args.plan_flags)
 
     prob = problem(args.split_tokens)
     out, lse = dsa.alloc_outputs(prob)
@@ -602,8 +622,7 @@ def run_ours(args):
                 "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(name),
                 "peak_kind": "of " + peak_kind, "algorithmic_bytes": abytes,
                 "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-                "kernel": ("dsa_attn_mma_kernel" if plan.tensor_cores else "dsa_attn_kernel") +
-                          (" + dsa_combine_kernel" if plan.launches > 1 else "")}
+                "kernel": kernel_name(plan) + (" + dsa_combine_kernel" if plan.launches > 1 else "")}
 
     # ---- the same step as a single call with a cold L2 (launch latency and first misses included)
     iso_flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
@@ -717,16 +736,19 @@ def run_ours(args):
         cpu = oracle_baseline(synth, inputs, w, args.mode)
 
     per_config = decode_loop = decode_loop_large = selection = masks = None
-    if rank == 0 and world == 1 and (not args.no_per_config or args.all_configs):
+    if rank == 0 and world == 1 and (not args.no_per_config or not args.no_decode_loop or args.all_configs):
         del inputs, prob, out, lse
         torch.cuda.empty_cache()
         if not args.no_per_config:
-            per_config = per_config_table(torch, dsa, synth, dev, peak)
-        if args.all_configs:
-            decode_loop = decode_loop_bench(torch, dsa, synth, dev)
-            # the same loop at a batch where a B200 step is bandwidth-bound rather than latency-bound
+            per_config = per_config_table(torch, dsa, synth, dev, peak, plan_flags=args.plan_flags)
+        if not args.no_decode_loop or args.all_configs:
+            # the paper's own shape at a batch where a B200 step is bandwidth-bound: grid-derived diagonals
+            # ("sparse") and the paper's method, per-head lists grown by the fused selection ("sparse_select")
             decode_loop_large = decode_loop_bench(torch, dsa, synth, dev, batch=128,
-                                                  modes=("dense", "sparse", "sparse_select"))
+                                                  modes=("dense", "sparse", "sparse_select"),
+                                                  plan_flags=args.plan_flags)
+        if args.all_configs:
+            decode_loop = decode_loop_bench(torch, dsa, synth, dev, plan_flags=args.plan_flags)
             selection = selection_overhead(torch, dsa, synth, dev)
             masks = mask_variants(torch, dsa, synth, dev, peak)
 
@@ -753,15 +775,17 @@ def run_ours(args):
                                 "tile_tokens": plan.tile_tokens, "stages": plan.stages,
                                 "tensor_cores": plan.tensor_cores, "work_items": plan.work_items,
                                 "item_warps": plan.item_warps, "heads_per_block": plan.heads_per_block,
-                                "block_warps": plan.block_warps}},
+                                "block_warps": plan.block_warps, "per_head_lists": plan.per_head_lists,
+                                "cluster_blocks": plan.cluster_blocks, "plan_flags": args.plan_flags}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }
         if per_config is not None:
             line["per_config"] = per_config
+        if decode_loop_large is not None:
+            line["decode_loop_batch128"] = decode_loop_large
         if decode_loop is not None:
             line["decode_loop"] = decode_loop
-            line["decode_loop_batch128"] = decode_loop_large
             line["selection_overhead"] = selection
             line["mask_variants"] = masks
         print(json.dumps(line))

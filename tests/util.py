@@ -9,7 +9,8 @@ from oracle import oracle as ora
 from paper_2609_19702_b200 import synth
 
 OUT_ATOL, OUT_RTOL, LSE_ATOL = 1e-2, 1e-2, 1e-3
-F32_ATOL, F32_RTOL, F32_LSE_ATOL = 2e-5, 2e-5, 2e-5
+# float32: the worst measured error is 4.4e-7 on the outputs and 9e-7 on the LSE (0.04 / 0.09 of these bounds)
+F32_ATOL, F32_RTOL, F32_LSE_ATOL = 1e-5, 1e-5, 1e-5
 
 
 def oracle_run(inp, mode, *, n_r=0, n_att=0, stride=0, trace=None, n_sink=0, want_kept=False, requests=None):
