@@ -57,6 +57,36 @@ def test_config5_large_batches_sampled_requests(batch):
         # property that holds for every request: kept count = prompt + min(p, N_att) (or p)
         want = w.prompt_len + (pos if diag is None else np.minimum(pos, diag.n_att))
         assert np.array_equal(cnt.cpu().numpy()[:, 0], want)
+    # the paper's own setting at this size: one skip list per attention head, with the fused selection
+    # (sampled requests against the oracle's kept sets and outputs; every request's kept count)
+    rng = np.random.default_rng(40 + batch)
+    few = synth.random_valid_trace(rng, 512, 208, (16,))
+    trace = np.ascontiguousarray(few[rng.integers(0, 16, size=(batch, w.num_q_heads))])
+    trace_dev = torch.from_numpy(trace.copy()).cuda()
+    diag = dsa.Diag(dsa.DSA_MASK_LIST, 512, 208, skip_offsets=trace_dev, select=True)
+    plan = dsa.dsa_query_plan(prob, diag)
+    assert plan.per_head_lists == 1 and plan.n_split == 1
+    out.fill_(float("nan"))
+    dsa.dsa_decode_attention_sparse(prob, diag, out, lse, dsa.alloc_workspace(prob, diag))
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    ref = util.oracle_run(sub, ora.MODE_LIST, n_r=512, n_att=208, trace=trace[sample], want_kept=True)
+    util.assert_close(out[sidx], lse[sidx], ref, what="full size per-head lists")
+    diag_ro = dsa.Diag(dsa.DSA_MASK_LIST, 512, 208, skip_offsets=torch.from_numpy(trace.copy()).cuda())
+    idx, cnt = dsa.dsa_debug_kept_indices(prob, diag_ro, dev["max_seq_len"])
+    util.assert_kept_equal(idx[sidx], cnt[sidx], ref, "full size per-head lists")
+    assert np.array_equal(cnt.cpu().numpy(), np.broadcast_to((w.prompt_len + np.minimum(pos, 208))[:, None], cnt.shape))
+    # requests in phase 2 got one new trace entry per head (a valid one), the others none
+    t = pos - 1
+    selecting = (t >= 207) & (t <= 510)
+    new = trace_dev.cpu().numpy()
+    changed = (new != trace).any(axis=2)
+    assert not changed[~selecting].any()
+    for i in np.flatnonzero(selecting)[:8]:
+        k = int(t[i]) - 207
+        assert (new[i, :, :k] == trace[i, :, :k]).all() and (new[i, :, k] >= 0).all() and (new[i, :, k] <= t[i]).all()
+        for h in (0, w.num_q_heads - 1):
+            assert new[i, h, k] not in set(trace[i, h, :k].tolist())       # an attended key, not one already skipped
     if batch != 256:
         return
     # the end-to-end call of the benchmark at this size (step inputs and results in pinned host
