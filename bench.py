@@ -91,7 +91,7 @@ def kernel_name(plan):
     if plan.per_head_lists:
         return "dsa_attn_heads_kernel"
     if plan.heads_per_block:
-        return "dsa_attn_group_kernel"
+        return "dsa_attn_gather_kernel" if plan.tensor_map_copies else "dsa_attn_group_kernel"
     return "dsa_attn_mma_kernel"
 
 
@@ -324,7 +324,7 @@ def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
                          "frac_of_peak": round(b_dense / t_dense / 1e9 / peak, 4),
                          "n_split": plan.n_split, "launches": plan.launches, "kernel": kernel_name(plan),
                          "heads_per_block": plan.heads_per_block, "item_warps": plan.item_warps,
-                         "cluster_blocks": plan.cluster_blocks},
+                         "cluster_blocks": plan.cluster_blocks, "tensor_map_copies": plan.tensor_map_copies},
                "sparse": []}
         for window, n_att in (windows or [(w.window, w.n_att)]):
             ww = synth.workload(w.index, batch=w.batch, window=window, n_att=n_att)
@@ -342,7 +342,8 @@ def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
                                   "ideal_byte_ratio": round(b_dense / b_sp, 3),
                                   "n_split": plan2.n_split, "launches": plan2.launches,
                                   "kernel": kernel_name(plan2), "heads_per_block": plan2.heads_per_block,
-                                  "item_warps": plan2.item_warps, "cluster_blocks": plan2.cluster_blocks})
+                                  "item_warps": plan2.item_warps, "cluster_blocks": plan2.cluster_blocks,
+                                  "tensor_map_copies": plan2.tensor_map_copies})
         rows.append(row)
         del inputs, prob, out, lse, ws
         torch.cuda.empty_cache()
@@ -776,7 +777,8 @@ def run_ours(args):
                                 "tensor_cores": plan.tensor_cores, "work_items": plan.work_items,
                                 "item_warps": plan.item_warps, "heads_per_block": plan.heads_per_block,
                                 "block_warps": plan.block_warps, "per_head_lists": plan.per_head_lists,
-                                "cluster_blocks": plan.cluster_blocks, "plan_flags": args.plan_flags}},
+                                "cluster_blocks": plan.cluster_blocks, "tensor_map_copies": plan.tensor_map_copies,
+                                "plan_flags": args.plan_flags}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }

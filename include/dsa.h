@@ -136,6 +136,9 @@ typedef struct dsa_problem {
 #define DSA_PLAN_NO_CLUSTER    0x80u  /* small launches: never let a thread-block cluster share a work item */
 #define DSA_PLAN_CLUSTER2      0x10000u /* small launches (several warps per item): clusters of 2 blocks  */
 #define DSA_PLAN_CLUSTER4      0x20000u /*                                           clusters of 4 blocks  */
+#define DSA_PLAN_GATHER        0x40000u /* head-group kernel, 4 warps: stage tiles by tensor-map gather copies */
+                                        /* (TMA, four scattered rows per copy) where the cache has a 2-D view */
+#define DSA_PLAN_NO_GATHER     0x80000u /* never do                                                        */
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u
 
@@ -213,12 +216,20 @@ typedef struct dsa_plan_info {
                             /* selection): shared tables per block, one candidate list per head    */
     int32_t cluster_blocks; /* blocks of a thread-block cluster that share one work item and merge */
                             /* through distributed shared memory (small launches); 1: no cluster   */
+    int32_t tensor_map_copies; /* 1: the head-group kernel stages its tiles with tensor-map gather  */
+                            /* copies (TMA) completing on mbarriers; 0: 16-byte cp.async copies    */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);
 DSA_API const char *dsa_status_string(int32_t status);
 /* CUDA error code recorded by the last failing call of this thread (0 if none). */
 DSA_API int32_t dsa_last_cuda_error(void);
+/* Number of bounded waits that gave up on the current device since the library was loaded.  The
+ * tensor-map kernel waits for each tile on an mbarrier for about a second at most; a copy that
+ * never lands makes it count here, stop waiting and run to its end, so that the context stays
+ * usable (the numbers of that call are then wrong).  0 in a healthy run.  count_out: host pointer.
+ * Synchronises with the device (a copy from a device symbol): not for use inside a capture. */
+DSA_API int32_t dsa_wait_timeouts(int32_t *count_out);
 
 /*
  * Configure every kernel variant of the library for the CURRENT device (a few hundred one-time

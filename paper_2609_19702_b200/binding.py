@@ -24,6 +24,7 @@ DSA_PLAN_CUDA_CORES, DSA_PLAN_NO_ITEM_WARPS, DSA_PLAN_RING_DEEP, DSA_PLAN_RING_S
 DSA_PLAN_GROUP, DSA_PLAN_NO_GROUP, DSA_PLAN_GROUP_W4 = 0x10, 0x20, 0x40
 DSA_PLAN_HEADS_PER_WARP_SHIFT = 8
 DSA_PLAN_NO_CLUSTER, DSA_PLAN_CLUSTER2, DSA_PLAN_CLUSTER4 = 0x80, 0x10000, 0x20000
+DSA_PLAN_GATHER, DSA_PLAN_NO_GATHER = 0x40000, 0x80000
 
 
 def plan_group(warps: int, heads_per_warp: int) -> int:
@@ -36,7 +37,8 @@ EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_works
            "dsa_query_plan", "dsa_decode_attention_dense", "dsa_decode_attention_sparse",
            "dsa_combine_splits", "dsa_debug_kept_indices",
            "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
-           "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len", "dsa_prepare"]
+           "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len", "dsa_prepare",
+           "dsa_wait_timeouts"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -70,7 +72,7 @@ class dsa_plan_info(ctypes.Structure):
                 ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32),
                 ("item_warps", ctypes.c_int32), ("heads_per_block", ctypes.c_int32),
                 ("block_warps", ctypes.c_int32), ("per_head_lists", ctypes.c_int32),
-                ("cluster_blocks", ctypes.c_int32)]
+                ("cluster_blocks", ctypes.c_int32), ("tensor_map_copies", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -97,6 +99,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_static_scratch.argtypes = [vp, vp, vp, vp, vp]
     lib.dsa_decode_attention_host_io.restype = i32
     lib.dsa_decode_attention_host_io.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.dsa_wait_timeouts.restype = i32
+    lib.dsa_wait_timeouts.argtypes = [ctypes.POINTER(i32)]
     lib.dsa_prepare.restype = i32
     lib.dsa_prepare.argtypes = []
     lib.dsa_decode_step.restype = i32
@@ -239,6 +243,13 @@ def dsa_prepare() -> None:
     """Configure every kernel variant for the current CUDA device (needed only before capturing
     calls that would otherwise be the first of their shape on this device)."""
     _check("dsa_prepare", _lib.dsa_prepare())
+
+
+def dsa_wait_timeouts() -> int:
+    """Bounded waits of the tensor-map kernel that gave up on the current device (0 in a healthy run)."""
+    n = ctypes.c_int32(0)
+    _check("dsa_wait_timeouts", _lib.dsa_wait_timeouts(ctypes.byref(n)))
+    return int(n.value)
 
 
 def dsa_query_plan(problem: Problem, diag: Optional[Diag] = None) -> dsa_plan_info:

@@ -45,7 +45,7 @@ int sm_count() {
 constexpr uint32_t kKnownPlanFlags = DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_RING_DEEP |
                                      DSA_PLAN_RING_SHALLOW | DSA_PLAN_GROUP | DSA_PLAN_NO_GROUP |
                                      DSA_PLAN_GROUP_W4 | DSA_PLAN_HEADS_PER_WARP_MASK | DSA_PLAN_NO_CLUSTER |
-                                     DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4;
+                                     DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4 | DSA_PLAN_GATHER | DSA_PLAN_NO_GATHER;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -69,6 +69,9 @@ struct Plan {
     int group_w;         // head-group tensor-core kernel: warps per block (0: not that kernel)
     int group_u;         // and kv heads each warp streams through the block's one row list
     int group_stages;    // and its ring depth
+    bool gather;         // and whether its tiles are staged by tensor-map gather copies; the 2-D cache view then:
+    int gather_rows_per_stride_b;
+    int64_t gather_rows; // its number of token rows
     bool heads;          // per-head-list tensor-core kernel (kHeadsWarps warps per block, group_u heads per warp)
     int dir_cap, kidx_cap;
     int64_t blocks;      // its grid
@@ -96,7 +99,7 @@ KernelQuery kernel_query(const Plan& pl) {
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
     q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
     q.mma_cl = pl.mma_cl;
-    q.group_w = pl.group_w; q.group_stages = pl.group_stages;
+    q.group_w = pl.group_w; q.group_stages = pl.group_stages; q.gather = pl.gather;
     q.heads = pl.heads; q.dir_cap = pl.dir_cap; q.kidx_cap = pl.kidx_cap; q.window = pl.window;
     return q;
 }
@@ -158,6 +161,25 @@ int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
 }
 
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// The K / V caches as a matrix [token rows][elements of one token row], which the tensor-map kernel
+// gathers rows of.  It exists when tokens are the outer dimension of a page / request (every head of a
+// token inside its token stride) and pages / requests start a whole number of token rows apart.
+bool gather_view(const dsa_problem* p, int* rows_per_stride_b, int64_t* rows) {
+    if (p->dtype != DSA_BF16 || p->head_dim % 64 != 0) return false;
+    const int64_t st = p->stride_token;
+    if (st <= 0 || (st * 2) % 16 != 0 || p->stride_batch % st != 0) return false;
+    if ((int64_t)(p->num_kv_heads - 1) * p->stride_head + p->head_dim > st) return false;
+    const int64_t rpb = p->stride_batch / st;
+    const int64_t units = p->block_table ? p->num_blocks : p->batch;
+    const int64_t last = p->block_table ? p->block_size : physical_capacity(p);
+    const int64_t n = (units - 1) * rpb + last;
+    if (units < 1 || last < 1 || rpb > 0x7fffffffLL || n < 1 || n >= 0x7fffffffLL) return false;
+    if (st > 0xffffffffLL || st * 2 >= (1LL << 40)) return false;      // (limits of a tensor map's extent and pitch)
+    *rows_per_stride_b = (int)rpb;
+    *rows = n;
+    return true;
+}
 
 // How many kv heads each warp of the head-group kernel should stream (a power of two), and with which
 // ring depth.
@@ -250,6 +272,9 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->group_w = 0;
     pl->group_u = 0;
     pl->group_stages = kGroupStages;
+    pl->gather = false;
+    pl->gather_rows_per_stride_b = 0;
+    pl->gather_rows = 0;
     pl->heads = false;
     pl->dir_cap = pl->kidx_cap = 0;
     pl->window = d ? d->window : 0;
@@ -384,6 +409,8 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
                 pl->group_w = w;
                 pl->group_u = u;
                 pl->group_stages = stages;
+                if (w == 4 && (p->plan_flags & DSA_PLAN_GATHER) && !(p->plan_flags & DSA_PLAN_NO_GATHER))
+                    pl->gather = gather_view(p, &pl->gather_rows_per_stride_b, &pl->gather_rows);
                 pl->mma_warps = 1;
                 pl->blocks = (int64_t)p->batch * pl->n_split * (p->num_kv_heads / (w * u));
             }
@@ -566,6 +593,71 @@ int32_t launch_combine(const float* out_part, const float* lse_part, int64_t row
 int32_t launch_append(const dsa_problem* problem, const void* k_new, const void* v_new, bool advance,
                       cudaStream_t st);
 
+// ---- tensor maps of the gather kernel --------------------------------------------------------------
+// Bounded waits of the gather kernel that gave up, per device (dsa_wait_timeouts reads it).
+__device__ int g_wait_timeouts;
+
+cudaError_t wait_timeouts_address(int** out) {
+    static std::atomic<int*> addr[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int* ptr = addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_wait_timeouts);
+        if (e != cudaSuccess) return e;
+        addr[dev].store(ptr, std::memory_order_release);
+    }
+    *out = ptr;
+    return cudaSuccess;
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link the driver).
+using TensorMapEncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+TensorMapEncodeFn tensor_map_encoder() {
+    static std::atomic<void*> cached{nullptr};
+    void* fn = cached.load(std::memory_order_acquire);
+    if (!fn) {
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess ||
+            qr != cudaDriverEntryPointSuccess || !fn) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        cached.store(fn, std::memory_order_release);
+    }
+    return reinterpret_cast<TensorMapEncodeFn>(fn);
+}
+
+// Views of the K and V caches for the plan's gather kernel: boxes of 64 elements (128 bytes) of one
+// row, which the gather4 copy stacks four at a time; 128-byte swizzle, so that the 8 rows an
+// ldmatrix reads lie in different banks.
+int32_t build_gather_maps(const dsa_problem* p, const Plan& pl, GatherMaps* g) {
+    const TensorMapEncodeFn encode = tensor_map_encoder();
+    if (!encode) return DSA_ERR_UNSUPPORTED;
+    const cuuint64_t dims[2] = {(cuuint64_t)((int64_t)(p->num_kv_heads - 1) * p->stride_head + p->head_dim),
+                                (cuuint64_t)pl.gather_rows};
+    const cuuint64_t pitch[1] = {(cuuint64_t)p->stride_token * 2};
+    const cuuint32_t box[2] = {64u, 1u};
+    const cuuint32_t step[2] = {1u, 1u};
+    for (int kv = 0; kv < 2; ++kv) {
+        const CUresult r = encode(kv ? &g->v : &g->k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                                  const_cast<void*>(kv ? p->v_cache : p->k_cache), dims, pitch, box, step,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return DSA_ERR_UNSUPPORTED;
+    }
+    g->rows_per_stride_b = pl.gather_rows_per_stride_b;
+    g->oob_row = (int)pl.gather_rows;
+    g->wait_timeouts = nullptr;
+    const cudaError_t e = wait_timeouts_address(&g->wait_timeouts);
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+}
+
 // k_new / v_new non-NULL: the fused decode step -- seq_len counts the tokens already cached, the
 // token being decoded is appended by this call and attended to as well.
 int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out, float* lse,
@@ -607,11 +699,16 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
             if (rc != DSA_OK) return rc;
         }
     }
+    GatherMaps maps;
+    if (pl.gather) {
+        rc = build_gather_maps(p, pl, &maps);
+        if (rc != DSA_OK) return rc;
+    }
     cudaError_t err = cudaSuccess;
     rc = dispatch(p->dtype, p->head_dim, [&](auto t, auto dd) -> int32_t {
         using T = decltype(t);
         err = kernel_launch<T, decltype(dd)::value>(kernel_query(pl), step && pl.mma, a, pl.grid, pl.smem, st,
-                                                    pl.blocks);
+                                                    pl.blocks, pl.gather ? &maps : nullptr);
         return DSA_OK;
     });
     if (rc != DSA_OK) return rc;
@@ -663,6 +760,15 @@ const char* dsa_status_string(int32_t status) {
 
 int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
 
+int32_t dsa_wait_timeouts(int32_t* count_out) {
+    if (!count_out) return DSA_ERR_INVALID_ARG;
+    int n = 0;
+    const cudaError_t e = cudaMemcpyFromSymbol(&n, g_wait_timeouts, sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(e);
+    *count_out = n;
+    return DSA_OK;
+}
+
 static cudaError_t static_scratch_address(void** out);
 
 int32_t dsa_prepare(void) {
@@ -699,6 +805,7 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->block_warps = pl.mma ? (block_warps > 0 ? block_warps : pl.mma_warps * pl.mma_kw) : 4;
     info->per_head_lists = pl.heads ? 1 : 0;
     info->cluster_blocks = pl.mma_cl;
+    info->tensor_map_copies = pl.gather ? 1 : 0;
     if (pl.mma_cl > 1) info->grid_blocks = (int32_t)(pl.grid * pl.mma_cl);
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;

@@ -3,6 +3,7 @@
 #pragma once
 #include "dsa_attn.cuh"
 #include "dsa_attn_mma.cuh"
+#include "dsa_attn_gather.cuh"
 #include "dsa_attn_group.cuh"
 #include "dsa_attn_heads.cuh"
 #include "dsa_launch.cuh"
@@ -157,6 +158,34 @@ struct KernelPick {
         return stages == kGroupStagesShallow ? launch_group_s<kGroupStagesShallow>(w, append, a, blocks, smem_bytes, st)
                                              : launch_group_s<kGroupStages>(w, append, a, blocks, smem_bytes, st);
     }
+    // The same with tensor-map gather copies (four-warp blocks).
+    static size_t smem_gather(int stages, int chunk, int bw) {
+        return stages == kGroupStagesShallow ? GatherCfg<D, 4, kGroupStagesShallow>::smem_bytes(chunk, bw)
+                                             : GatherCfg<D, 4, kGroupStages>::smem_bytes(chunk, bw);
+    }
+    template <bool APPEND, int ST>
+    static ConfiguredFlags* gather_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    template <bool APPEND, int ST>
+    static cudaError_t launch_gather_s(const AttnArgs& a, const GatherMaps& maps, int64_t blocks, size_t smem_bytes,
+                                       cudaStream_t st) {
+        if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            auto kern = dsa_attn_gather_kernel<D, G, ST, 4, APPEND>;
+            const cudaError_t e = ensure_configured(kern, gather_configured<APPEND, ST>());
+            if (e != cudaSuccess) return e;
+            return launch_pdl(kern, (unsigned)blocks, 32 * 4, smem_bytes, st, a, maps);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
+    static cudaError_t launch_gather(int stages, bool append, const AttnArgs& a, const GatherMaps* maps, int64_t blocks,
+                                     size_t smem_bytes, cudaStream_t st) {
+        if (!maps) return cudaErrorInvalidValue;
+        if (stages == kGroupStagesShallow)
+            return append ? launch_gather_s<true, kGroupStagesShallow>(a, *maps, blocks, smem_bytes, st)
+                          : launch_gather_s<false, kGroupStagesShallow>(a, *maps, blocks, smem_bytes, st);
+        return append ? launch_gather_s<true, kGroupStages>(a, *maps, blocks, smem_bytes, st)
+                      : launch_gather_s<false, kGroupStages>(a, *maps, blocks, smem_bytes, st);
+    }
     // Per-head-list tensor-core kernel (bf16, list masks per kv or query head, fused selection).
     static size_t smem_heads(int dir_cap, int window, int kidx_cap, int bw) {
         return HeadsCfg<D, G, kMmaStages, kHeadsWarps, HM>::smem_bytes(dir_cap, window, kidx_cap, bw);
@@ -229,6 +258,16 @@ struct KernelPick {
                 group(two{}, std::true_type{}, gshallow{});
                 group(four{}, std::false_type{}, gshallow{});
                 group(four{}, std::true_type{}, gshallow{});
+                auto gather = [&](auto app, auto stg) {
+                    constexpr int ST = decltype(stg)::value;
+                    constexpr bool APPEND = decltype(app)::value;
+                    if (e == cudaSuccess)
+                        e = ensure_configured(dsa_attn_gather_kernel<D, G, ST, 4, APPEND>, gather_configured<APPEND, ST>());
+                };
+                gather(std::false_type{}, gdeep{});
+                gather(std::true_type{}, gdeep{});
+                gather(std::false_type{}, gshallow{});
+                gather(std::true_type{}, gshallow{});
                 mma(two{}, std::false_type{}, one{}, deep{});
                 mma(two{}, std::true_type{}, one{}, deep{});
                 mma(two{}, std::false_type{}, one{}, shallow{});
@@ -297,7 +336,8 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
         }
         if (q.mma && q.group_w > 0) {
             out->stages = q.group_stages == kGroupStagesShallow ? kGroupStagesShallow : kGroupStages;
-            out->smem = P::smem_group(q.group_w, out->stages, chunk, bitmap_words);
+            out->smem = q.gather ? P::smem_gather(out->stages, chunk, bitmap_words)
+                                 : P::smem_group(q.group_w, out->stages, chunk, bitmap_words);
             return;
         }
         const bool shallow = q.mma && q.mma_stages == kMmaStagesShallow && q.mma_warps == 2 && q.mma_kw == 1 &&
@@ -310,12 +350,13 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
 
 template <typename T, int D>
 cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
-                          cudaStream_t st, int64_t blocks) {
+                          cudaStream_t st, int64_t blocks, const GatherMaps* maps) {
     cudaError_t err = cudaErrorInvalidValue;
     dispatch_variant<T, D>(q, [&](auto pick) {
         using P = decltype(pick);
         if (q.mma && q.mma_kw > 1 && q.mma_cl > 1) err = P::launch_cluster(q.mma_cl, append, a, items, smem, st);
         else if (q.mma && q.heads) err = P::launch_heads(append, a, blocks, smem, st);
+        else if (q.mma && q.group_w > 0 && q.gather) err = P::launch_gather(q.group_stages, append, a, maps, blocks, smem, st);
         else if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
         else
         err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, q.mma_stages, a, items, smem, st, append)

@@ -3,6 +3,6 @@
 
 namespace dsa {
 template bool kernel_shape<__nv_bfloat16, 64>(const KernelQuery&, int, int, KernelShape*);
-template cudaError_t kernel_launch<__nv_bfloat16, 64>(const KernelQuery&, bool, const AttnArgs&, int64_t, size_t, cudaStream_t, int64_t);
+template cudaError_t kernel_launch<__nv_bfloat16, 64>(const KernelQuery&, bool, const AttnArgs&, int64_t, size_t, cudaStream_t, int64_t, const GatherMaps*);
 template cudaError_t kernel_prepare<__nv_bfloat16, 64>();
 }  // namespace dsa

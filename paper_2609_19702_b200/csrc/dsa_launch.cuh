@@ -29,6 +29,7 @@ struct KernelQuery {
     int group_w;             // head-group tensor-core kernel: warps per block that share one row list for
                              // group_w x heads_per_warp kv heads (2 or 4); 0: not that kernel
     int group_stages;        // its ring depth: kGroupStages or kGroupStagesShallow
+    bool gather;             // head-group kernel whose tiles are staged by tensor-map gather copies (group_w 4)
     bool heads;              // per-head-list tensor-core kernel (blocks of kHeadsWarps warps); sizes of its tables:
     int dir_cap, kidx_cap, window;
 };
@@ -45,10 +46,11 @@ bool kernel_shape(const KernelQuery& q, int chunk, int bitmap_words, KernelShape
 
 // Launch it: `items` (request, kv head, split) work items; `append`: the fused decode step (the
 // kernel reads the current token's rows from a.k_new / a.v_new and stores them to the cache);
-// `blocks`: thread blocks of the head-group kernel (ignored by the others).
+// `blocks`: thread blocks of the head-group kernel (ignored by the others); `maps`: the cache views
+// of the tensor-map form of it (q.gather), NULL otherwise.
 template <typename T, int D>
 cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, int64_t items, size_t smem,
-                          cudaStream_t st, int64_t blocks);
+                          cudaStream_t st, int64_t blocks, const GatherMaps* maps);
 
 // Configure every variant of (T, D) for the current device, so that no later launch has to (a
 // launch inside a stream capture must not).

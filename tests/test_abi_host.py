@@ -36,6 +36,13 @@ def test_every_declared_symbol_is_exported(dsa):
         assert hasattr(dsa, n) or n in ("dsa_status_string", "dsa_last_cuda_error"), n
 
 
+def test_wait_timeouts_validates_its_argument(dsa):
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    lib.dsa_wait_timeouts.restype = ctypes.c_int32
+    lib.dsa_wait_timeouts.argtypes = [ctypes.c_void_p]
+    assert lib.dsa_wait_timeouts(None) == -1
+
+
 def test_version_and_status_strings(dsa):
     assert dsa.dsa_version() == 100
     lib = ctypes.CDLL(dsa.LIB_PATH)
@@ -183,6 +190,30 @@ def test_newer_entry_points_validate_before_touching_a_device(dsa):
     host_io = lib.dsa_decode_attention_host_io
     host_io.argtypes = [ctypes.c_void_p] * 11 + [ctypes.c_size_t, ctypes.c_void_p]
     assert host_io(ctypes.byref(p), ctypes.byref(d), None, hp, hp, None, fake, fake, hp, hp, None, 0, None) == -1
+
+
+def test_tensor_map_copies_only_on_request_and_only_with_a_2d_view(dsa):
+    big = dict(batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360, max_prompt_len=200,
+               stride_batch=4360 * 4096, stride_token=4096, stride_head=128)
+    diag = _diag(dsa, window=512, n_att=208, grid_w=64)
+    rc, info = _plan(dsa, _problem(dsa, **big), diag)
+    assert rc == 0 and info.heads_per_block > 0 and info.tensor_map_copies == 0      # never by itself
+    rc, info = _plan(dsa, _problem(dsa, plan_flags=dsa.DSA_PLAN_GATHER, **big), diag)
+    assert rc == 0 and info.tensor_map_copies == 1 and info.block_warps == 4
+    rc, info = _plan(dsa, _problem(dsa, plan_flags=dsa.DSA_PLAN_GATHER | dsa.DSA_PLAN_NO_GATHER, **big), diag)
+    assert rc == 0 and info.tensor_map_copies == 0
+    # head-major cache (a head's tokens contiguous): rows of different heads are not columns of one matrix
+    head_major = dict(big, stride_batch=32 * 4360 * 128, stride_token=128, stride_head=4360 * 128)
+    rc, info = _plan(dsa, _problem(dsa, plan_flags=dsa.DSA_PLAN_GATHER, **head_major), diag)
+    assert rc == 0 and info.tensor_map_copies == 0
+    # requests that do not start a whole number of token rows apart
+    rc, info = _plan(dsa, _problem(dsa, plan_flags=dsa.DSA_PLAN_GATHER, **dict(big, stride_batch=4360 * 4096 + 8)), diag)
+    assert rc == 0 and info.tensor_map_copies == 0
+    # float32 and the two-warp head-group form have no such kernel
+    rc, info = _plan(dsa, _problem(dsa, dtype=dsa.DSA_F32, plan_flags=dsa.DSA_PLAN_GATHER, **big), diag)
+    assert rc == 0 and info.tensor_map_copies == 0
+    rc, info = _plan(dsa, _problem(dsa, plan_flags=dsa.plan_group(2, 1) | dsa.DSA_PLAN_GATHER, **big), diag)
+    assert rc == 0 and info.block_warps == 2 and info.tensor_map_copies == 0
 
 
 def test_ring_depth_follows_the_wave_estimate(dsa):

@@ -22,7 +22,8 @@ from tests import test_gpu_selection as t_sel
 
 pytestmark = pytest.mark.gpu
 
-SHAPES = [(2, 1), (4, 1), (2, 2), (4, 2), (2, 4)]
+# (warps per block, kv heads per warp, tiles staged by tensor-map gather copies)
+SHAPES = [(2, 1, False), (4, 1, False), (2, 2, False), (4, 2, False), (2, 4, False), (4, 1, True), (4, 2, True)]
 
 
 @pytest.fixture(scope="module")
@@ -31,11 +32,11 @@ def dsa():
     return binding
 
 
-@pytest.fixture(params=SHAPES, ids=["w%du%d" % s for s in SHAPES])
+@pytest.fixture(params=SHAPES, ids=["w%du%d%s" % (w, u, "tma" if tma else "") for w, u, tma in SHAPES])
 def forced(request, dsa, monkeypatch):
     """Every problem handed to the library carries the head-group switch."""
-    w, u = request.param
-    flags = dsa.plan_group(w, u)
+    w, u, tma = request.param
+    flags = dsa.plan_group(w, u) | (dsa.DSA_PLAN_GATHER if tma else dsa.DSA_PLAN_NO_GATHER)
     orig = dsa.Problem.c_struct
 
     def patched(self):
@@ -48,7 +49,7 @@ def forced(request, dsa, monkeypatch):
 
 
 def test_the_switch_really_selects_the_head_group_kernel(dsa, forced):
-    w_, u_ = forced
+    w_, u_, tma_ = forced
     for w in (synth.workload(5, batch=2), synth.workload(4, batch=2), synth.workload(2, batch=4)):
         inp = synth.make_inputs(w)
         prob = dsa.problem_from_host(inp)
@@ -60,6 +61,8 @@ def test_the_switch_really_selects_the_head_group_kernel(dsa, forced):
             if w.num_kv_heads % (w_ * u_) == 0:
                 assert plan.heads_per_block == w_ * u_ and plan.block_warps == w_ and plan.tensor_cores == 1
                 assert plan.grid_blocks * w_ * u_ == plan.work_items and plan.item_warps == 1
+                # (all three workloads keep tokens outermost, so the caches have the 2-D view)
+                assert plan.tensor_map_copies == (1 if tma_ else 0)
             else:
                 assert plan.heads_per_block == 0
         # one mask per query head, with and without the fused selection: the per-head-list kernel (4 warps)
@@ -79,6 +82,12 @@ def test_the_switch_really_selects_the_head_group_kernel(dsa, forced):
     w = synth.workload(1)
     prob = dsa.problem_from_host(synth.make_inputs(w), dtype=torch.float32)
     assert dsa.dsa_query_plan(prob, None).heads_per_block == 0
+
+
+def test_no_wait_ever_gave_up(dsa):
+    """The tensor-map kernel bounds its mbarrier waits and counts the ones that ran out."""
+    torch.cuda.synchronize()
+    assert dsa.dsa_wait_timeouts() == 0
 
 
 def test_five_configurations(dsa, forced):
