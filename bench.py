@@ -91,7 +91,9 @@ def kernel_name(plan):
     if plan.per_head_lists:
         return "dsa_attn_heads_kernel"
     if plan.heads_per_block:
-        return "dsa_attn_gather_kernel" if plan.tensor_map_copies else "dsa_attn_group_kernel"
+        if plan.tensor_map_copies:
+            return "dsa_attn_gather_kernel"
+        return "dsa_attn_group_ws_kernel" if plan.producer_warps else "dsa_attn_group_kernel"
     return "dsa_attn_mma_kernel"
 
 
@@ -324,7 +326,8 @@ def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
                          "frac_of_peak": round(b_dense / t_dense / 1e9 / peak, 4),
                          "n_split": plan.n_split, "launches": plan.launches, "kernel": kernel_name(plan),
                          "heads_per_block": plan.heads_per_block, "item_warps": plan.item_warps,
-                         "cluster_blocks": plan.cluster_blocks, "tensor_map_copies": plan.tensor_map_copies},
+                         "cluster_blocks": plan.cluster_blocks, "tensor_map_copies": plan.tensor_map_copies,
+                         "producer_warps": plan.producer_warps},
                "sparse": []}
         for window, n_att in (windows or [(w.window, w.n_att)]):
             ww = synth.workload(w.index, batch=w.batch, window=window, n_att=n_att)
@@ -343,7 +346,8 @@ def per_config_table(torch, dsa, synth, dev, peak, plan_flags=0, only=None):
                                   "n_split": plan2.n_split, "launches": plan2.launches,
                                   "kernel": kernel_name(plan2), "heads_per_block": plan2.heads_per_block,
                                   "item_warps": plan2.item_warps, "cluster_blocks": plan2.cluster_blocks,
-                                  "tensor_map_copies": plan2.tensor_map_copies})
+                                  "tensor_map_copies": plan2.tensor_map_copies,
+                                  "producer_warps": plan2.producer_warps})
         rows.append(row)
         del inputs, prob, out, lse, ws
         torch.cuda.empty_cache()
@@ -778,7 +782,7 @@ def run_ours(args):
                                 "item_warps": plan.item_warps, "heads_per_block": plan.heads_per_block,
                                 "block_warps": plan.block_warps, "per_head_lists": plan.per_head_lists,
                                 "cluster_blocks": plan.cluster_blocks, "tensor_map_copies": plan.tensor_map_copies,
-                                "plan_flags": args.plan_flags}},
+                                "producer_warps": plan.producer_warps, "plan_flags": args.plan_flags}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": plan.launches * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "variants": variants,
         }

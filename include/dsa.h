@@ -139,6 +139,8 @@ typedef struct dsa_problem {
 #define DSA_PLAN_GATHER        0x40000u /* head-group kernel, 4 warps: stage tiles by tensor-map gather copies */
                                         /* (TMA, four scattered rows per copy) where the cache has a 2-D view */
 #define DSA_PLAN_NO_GATHER     0x80000u /* never do                                                        */
+#define DSA_PLAN_PRODUCERS     0x100000u /* head-group kernel, 4 warps: a producer warp beside every consumer warp */
+#define DSA_PLAN_NO_PRODUCERS  0x200000u /* never                                                       */
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u
 
@@ -218,6 +220,8 @@ typedef struct dsa_plan_info {
                             /* through distributed shared memory (small launches); 1: no cluster   */
     int32_t tensor_map_copies; /* 1: the head-group kernel stages its tiles with tensor-map gather  */
                             /* copies (TMA) completing on mbarriers; 0: 16-byte cp.async copies    */
+    int32_t producer_warps; /* warps per block that only issue copies (one per consumer warp, handing */
+                            /* tiles over through mbarriers); 0: every warp copies and computes       */
 } dsa_plan_info;
 
 DSA_API int32_t dsa_version(void);

@@ -25,6 +25,7 @@ DSA_PLAN_GROUP, DSA_PLAN_NO_GROUP, DSA_PLAN_GROUP_W4 = 0x10, 0x20, 0x40
 DSA_PLAN_HEADS_PER_WARP_SHIFT = 8
 DSA_PLAN_NO_CLUSTER, DSA_PLAN_CLUSTER2, DSA_PLAN_CLUSTER4 = 0x80, 0x10000, 0x20000
 DSA_PLAN_GATHER, DSA_PLAN_NO_GATHER = 0x40000, 0x80000
+DSA_PLAN_PRODUCERS, DSA_PLAN_NO_PRODUCERS = 0x100000, 0x200000
 
 
 def plan_group(warps: int, heads_per_warp: int) -> int:
@@ -72,7 +73,8 @@ class dsa_plan_info(ctypes.Structure):
                 ("stages", ctypes.c_int32), ("tensor_cores", ctypes.c_int32), ("work_items", ctypes.c_int32),
                 ("item_warps", ctypes.c_int32), ("heads_per_block", ctypes.c_int32),
                 ("block_warps", ctypes.c_int32), ("per_head_lists", ctypes.c_int32),
-                ("cluster_blocks", ctypes.c_int32), ("tensor_map_copies", ctypes.c_int32)]
+                ("cluster_blocks", ctypes.c_int32), ("tensor_map_copies", ctypes.c_int32),
+                ("producer_warps", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:

@@ -45,7 +45,8 @@ int sm_count() {
 constexpr uint32_t kKnownPlanFlags = DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARPS | DSA_PLAN_RING_DEEP |
                                      DSA_PLAN_RING_SHALLOW | DSA_PLAN_GROUP | DSA_PLAN_NO_GROUP |
                                      DSA_PLAN_GROUP_W4 | DSA_PLAN_HEADS_PER_WARP_MASK | DSA_PLAN_NO_CLUSTER |
-                                     DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4 | DSA_PLAN_GATHER | DSA_PLAN_NO_GATHER;
+                                     DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4 | DSA_PLAN_GATHER | DSA_PLAN_NO_GATHER | DSA_PLAN_PRODUCERS |
+                                     DSA_PLAN_NO_PRODUCERS;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -69,6 +70,7 @@ struct Plan {
     int group_w;         // head-group tensor-core kernel: warps per block (0: not that kernel)
     int group_u;         // and kv heads each warp streams through the block's one row list
     int group_stages;    // and its ring depth
+    bool producers;      // and whether every ring has a producer warp beside its consumer warp
     bool gather;         // and whether its tiles are staged by tensor-map gather copies; the 2-D cache view then:
     int gather_rows_per_stride_b;
     int64_t gather_rows; // its number of token rows
@@ -99,7 +101,7 @@ KernelQuery kernel_query(const Plan& pl) {
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
     q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
     q.mma_cl = pl.mma_cl;
-    q.group_w = pl.group_w; q.group_stages = pl.group_stages; q.gather = pl.gather;
+    q.group_w = pl.group_w; q.group_stages = pl.group_stages; q.gather = pl.gather; q.producers = pl.producers;
     q.heads = pl.heads; q.dir_cap = pl.dir_cap; q.kidx_cap = pl.kidx_cap; q.window = pl.window;
     return q;
 }
@@ -273,6 +275,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->group_u = 0;
     pl->group_stages = kGroupStages;
     pl->gather = false;
+    pl->producers = false;
     pl->gather_rows_per_stride_b = 0;
     pl->gather_rows = 0;
     pl->heads = false;
@@ -411,6 +414,15 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
                 pl->group_stages = stages;
                 if (w == 4 && (p->plan_flags & DSA_PLAN_GATHER) && !(p->plan_flags & DSA_PLAN_NO_GATHER))
                     pl->gather = gather_view(p, &pl->gather_rows_per_stride_b, &pl->gather_rows);
+                // Producer warps pay where the grid is more than one wave of deep-ring blocks (measured on the
+                // paged workload: batch 224 / 256, 1.5 / 1.7 waves: -3.5 % / -1.7 %; window 1024: -1.4 %), not
+                // where all blocks are resident from the start (batch 32 ... 128: +2 ... 3 %), and with the
+                // shallow ring they cannot run three blocks to an SM at all (registers).
+                const int64_t n_blocks = (int64_t)p->batch * pl->n_split * (p->num_kv_heads / (w * u));
+                const bool pays = stages == kGroupStages && pl->n_split == 1 && n_blocks > 2 * (int64_t)kNumSMs;
+                if (w == 4 && !pl->gather && !(p->plan_flags & DSA_PLAN_NO_PRODUCERS) &&
+                    ((p->plan_flags & DSA_PLAN_PRODUCERS) || pays))
+                    pl->producers = true;
                 pl->mma_warps = 1;
                 pl->blocks = (int64_t)p->batch * pl->n_split * (p->num_kv_heads / (w * u));
             }
@@ -550,6 +562,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->out = nullptr; a->lse = nullptr; a->out_part = nullptr; a->lse_part = nullptr;
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
     a->step_append = 0; a->k_new = nullptr; a->v_new = nullptr;
+    a->wait_timeouts = nullptr;
 }
 
 // `after_attention`: the combine follows the attention kernel of the same call.  It is then
@@ -653,9 +666,7 @@ int32_t build_gather_maps(const dsa_problem* p, const Plan& pl, GatherMaps* g) {
     }
     g->rows_per_stride_b = pl.gather_rows_per_stride_b;
     g->oob_row = (int)pl.gather_rows;
-    g->wait_timeouts = nullptr;
-    const cudaError_t e = wait_timeouts_address(&g->wait_timeouts);
-    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+    return DSA_OK;
 }
 
 // k_new / v_new non-NULL: the fused decode step -- seq_len counts the tokens already cached, the
@@ -698,6 +709,10 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
             rc = launch_append(p, k_new, v_new, false, st);
             if (rc != DSA_OK) return rc;
         }
+    }
+    if (pl.gather || pl.producers) {                  // (the kernels with bounded mbarrier waits)
+        const cudaError_t e = wait_timeouts_address(&a.wait_timeouts);
+        if (e != cudaSuccess) return cuda_fail(e);
     }
     GatherMaps maps;
     if (pl.gather) {
@@ -806,6 +821,7 @@ int32_t dsa_query_plan(const dsa_problem* problem, const dsa_diag_params* diag, 
     info->per_head_lists = pl.heads ? 1 : 0;
     info->cluster_blocks = pl.mma_cl;
     info->tensor_map_copies = pl.gather ? 1 : 0;
+    info->producer_warps = pl.producers ? pl.group_w : 0;
     if (pl.mma_cl > 1) info->grid_blocks = (int32_t)(pl.grid * pl.mma_cl);
     info->smem_bytes = (int32_t)pl.smem;
     info->tile_tokens = pl.tile;

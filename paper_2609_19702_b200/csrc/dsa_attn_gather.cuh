@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_gather_kernel(const AttnArgs 
                     while (!mbar_try_wait(bars + cslot, parity)) {
                         if (clock64() - t0 > kGatherWaitCycles) { gave_up = true; break; }
                     }
-                    if (gave_up && lane == 0 && g.wait_timeouts) atomicAdd(g.wait_timeouts, 1);
+                    if (gave_up && lane == 0 && a.wait_timeouts) atomicAdd(a.wait_timeouts, 1);
                 }
             }
             phases ^= 1u << cslot;

@@ -49,6 +49,7 @@ struct AttnArgs {
     int step_append;             // 0: seq_len counts the current token, nothing is appended
     const void* k_new;           // [B, H_kv, D] rows of the current token; NULL: already in the cache
     const void* v_new;
+    int* wait_timeouts;          // device counter of bounded mbarrier waits that gave up (0 in a healthy run); may be NULL
 };
 
 // What the tensor-map (gather) kernel needs beyond AttnArgs: the K and V caches as 2-D views
@@ -57,7 +58,6 @@ struct GatherMaps {
     CUtensorMap k, v;
     int rows_per_stride_b;       // token rows between neighbouring pages (paged cache) or requests
     int oob_row;                 // a row index beyond the view: such a row reads as zeros
-    int* wait_timeouts;          // device counter of bounded waits that gave up (0 in a healthy run); may be NULL
 };
 
 // The prompt length of request b as the kernels use it.  With a bounded cache a request's region

@@ -4,6 +4,7 @@
 #include "dsa_attn.cuh"
 #include "dsa_attn_mma.cuh"
 #include "dsa_attn_gather.cuh"
+#include "dsa_attn_group_ws.cuh"
 #include "dsa_attn_group.cuh"
 #include "dsa_attn_heads.cuh"
 #include "dsa_launch.cuh"
@@ -186,6 +187,29 @@ struct KernelPick {
         return append ? launch_gather_s<true, kGroupStages>(a, *maps, blocks, smem_bytes, st)
                       : launch_gather_s<false, kGroupStages>(a, *maps, blocks, smem_bytes, st);
     }
+    // The same with a producer warp per ring (four consumer + four producer warps; the shared memory of
+    // the plain four-warp form).
+    template <bool APPEND, int ST>
+    static ConfiguredFlags* ws_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    template <bool APPEND, int ST>
+    static cudaError_t launch_ws_s(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
+        if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            auto kern = dsa_attn_group_ws_kernel<D, G, ST, 4, APPEND>;
+            const cudaError_t e = ensure_configured(kern, ws_configured<APPEND, ST>());
+            if (e != cudaSuccess) return e;
+            return launch_pdl(kern, (unsigned)blocks, 64 * 4, smem_bytes, st, a);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    }
+    static cudaError_t launch_ws(int stages, bool append, const AttnArgs& a, int64_t blocks, size_t smem_bytes,
+                                 cudaStream_t st) {
+        if (stages == kGroupStagesShallow)
+            return append ? launch_ws_s<true, kGroupStagesShallow>(a, blocks, smem_bytes, st)
+                          : launch_ws_s<false, kGroupStagesShallow>(a, blocks, smem_bytes, st);
+        return append ? launch_ws_s<true, kGroupStages>(a, blocks, smem_bytes, st)
+                      : launch_ws_s<false, kGroupStages>(a, blocks, smem_bytes, st);
+    }
     // Per-head-list tensor-core kernel (bf16, list masks per kv or query head, fused selection).
     static size_t smem_heads(int dir_cap, int window, int kidx_cap, int bw) {
         return HeadsCfg<D, G, kMmaStages, kHeadsWarps, HM>::smem_bytes(dir_cap, window, kidx_cap, bw);
@@ -264,6 +288,16 @@ struct KernelPick {
                     if (e == cudaSuccess)
                         e = ensure_configured(dsa_attn_gather_kernel<D, G, ST, 4, APPEND>, gather_configured<APPEND, ST>());
                 };
+                auto ws = [&](auto app, auto stg) {
+                    constexpr int ST = decltype(stg)::value;
+                    constexpr bool APPEND = decltype(app)::value;
+                    if (e == cudaSuccess)
+                        e = ensure_configured(dsa_attn_group_ws_kernel<D, G, ST, 4, APPEND>, ws_configured<APPEND, ST>());
+                };
+                ws(std::false_type{}, gdeep{});
+                ws(std::true_type{}, gdeep{});
+                ws(std::false_type{}, gshallow{});
+                ws(std::true_type{}, gshallow{});
                 gather(std::false_type{}, gdeep{});
                 gather(std::true_type{}, gdeep{});
                 gather(std::false_type{}, gshallow{});
@@ -356,6 +390,7 @@ cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, 
         using P = decltype(pick);
         if (q.mma && q.mma_kw > 1 && q.mma_cl > 1) err = P::launch_cluster(q.mma_cl, append, a, items, smem, st);
         else if (q.mma && q.heads) err = P::launch_heads(append, a, blocks, smem, st);
+        else if (q.mma && q.group_w > 0 && q.producers) err = P::launch_ws(q.group_stages, append, a, blocks, smem, st);
         else if (q.mma && q.group_w > 0 && q.gather) err = P::launch_gather(q.group_stages, append, a, maps, blocks, smem, st);
         else if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
         else

@@ -30,6 +30,7 @@ struct KernelQuery {
                              // group_w x heads_per_warp kv heads (2 or 4); 0: not that kernel
     int group_stages;        // its ring depth: kGroupStages or kGroupStagesShallow
     bool gather;             // head-group kernel whose tiles are staged by tensor-map gather copies (group_w 4)
+    bool producers;          // head-group kernel with a producer warp beside every consumer warp (group_w 4)
     bool heads;              // per-head-list tensor-core kernel (blocks of kHeadsWarps warps); sizes of its tables:
     int dir_cap, kidx_cap, window;
 };

@@ -216,6 +216,30 @@ def test_tensor_map_copies_only_on_request_and_only_with_a_2d_view(dsa):
     assert rc == 0 and info.block_warps == 2 and info.tensor_map_copies == 0
 
 
+def test_producer_warps_only_for_grids_of_more_than_one_wave(dsa):
+    shape = dict(num_q_heads=32, num_kv_heads=32, max_seq_len=4360, max_prompt_len=200,
+                 stride_batch=4360 * 4096, stride_token=4096, stride_head=128)
+    diag = _diag(dsa, window=512, n_att=208, grid_w=64)
+
+    def plan(batch, flags=0, d=diag):
+        rc, info = _plan(dsa, _problem(dsa, batch=batch, plan_flags=flags, **shape), d)
+        assert rc == 0
+        return info
+    big = plan(256)                       # 512 deep-ring blocks on 296 slots
+    assert big.block_warps == 4 and big.stages == 3 and big.grid_blocks > 296 and big.producer_warps == 4
+    assert plan(256, dsa.DSA_PLAN_NO_PRODUCERS).producer_warps == 0
+    small = plan(128)                     # every block resident from the start
+    assert small.grid_blocks <= 296 and small.producer_warps == 0
+    assert plan(128, dsa.DSA_PLAN_PRODUCERS).producer_warps == 4
+    shallow = plan(192)                   # three blocks to an SM: the registers of 8 warps a block do not fit
+    assert shallow.stages == 2 and shallow.producer_warps == 0
+    dense = plan(256, d=None)             # split plans keep the plain form
+    assert dense.n_split > 1 and dense.producer_warps == 0
+    # the tensor-map form has no producer warps, and the two-warp head-group form neither
+    assert plan(256, dsa.DSA_PLAN_GATHER).producer_warps == 0
+    assert plan(256, dsa.plan_group(2, 1) | dsa.DSA_PLAN_PRODUCERS).producer_warps == 0
+
+
 def test_ring_depth_follows_the_wave_estimate(dsa):
     def stages(batch):
         rc, info = _plan(dsa, _problem(dsa, batch=batch, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,

@@ -22,8 +22,10 @@ from tests import test_gpu_selection as t_sel
 
 pytestmark = pytest.mark.gpu
 
-# (warps per block, kv heads per warp, tiles staged by tensor-map gather copies)
-SHAPES = [(2, 1, False), (4, 1, False), (2, 2, False), (4, 2, False), (2, 4, False), (4, 1, True), (4, 2, True)]
+# (warps per block, kv heads per warp, form: "" cp.async by the computing warps, "tma" tensor-map gather
+# copies, "ws" producer warps)
+SHAPES = [(2, 1, ""), (4, 1, ""), (2, 2, ""), (4, 2, ""), (2, 4, ""), (4, 1, "tma"), (4, 2, "tma"), (4, 1, "ws"),
+          (4, 2, "ws")]
 
 
 @pytest.fixture(scope="module")
@@ -32,11 +34,12 @@ def dsa():
     return binding
 
 
-@pytest.fixture(params=SHAPES, ids=["w%du%d%s" % (w, u, "tma" if tma else "") for w, u, tma in SHAPES])
+@pytest.fixture(params=SHAPES, ids=["w%du%d%s" % s for s in SHAPES])
 def forced(request, dsa, monkeypatch):
     """Every problem handed to the library carries the head-group switch."""
-    w, u, tma = request.param
-    flags = dsa.plan_group(w, u) | (dsa.DSA_PLAN_GATHER if tma else dsa.DSA_PLAN_NO_GATHER)
+    w, u, form = request.param
+    flags = dsa.plan_group(w, u) | (dsa.DSA_PLAN_GATHER if form == "tma" else dsa.DSA_PLAN_NO_GATHER) | \
+        (dsa.DSA_PLAN_PRODUCERS if form == "ws" else dsa.DSA_PLAN_NO_PRODUCERS)
     orig = dsa.Problem.c_struct
 
     def patched(self):
@@ -49,7 +52,7 @@ def forced(request, dsa, monkeypatch):
 
 
 def test_the_switch_really_selects_the_head_group_kernel(dsa, forced):
-    w_, u_, tma_ = forced
+    w_, u_, form_ = forced
     for w in (synth.workload(5, batch=2), synth.workload(4, batch=2), synth.workload(2, batch=4)):
         inp = synth.make_inputs(w)
         prob = dsa.problem_from_host(inp)
@@ -62,7 +65,8 @@ def test_the_switch_really_selects_the_head_group_kernel(dsa, forced):
                 assert plan.heads_per_block == w_ * u_ and plan.block_warps == w_ and plan.tensor_cores == 1
                 assert plan.grid_blocks * w_ * u_ == plan.work_items and plan.item_warps == 1
                 # (all three workloads keep tokens outermost, so the caches have the 2-D view)
-                assert plan.tensor_map_copies == (1 if tma_ else 0)
+                assert plan.tensor_map_copies == (1 if form_ == "tma" else 0)
+                assert plan.producer_warps == (4 if form_ == "ws" else 0)
             else:
                 assert plan.heads_per_block == 0
         # one mask per query head, with and without the fused selection: the per-head-list kernel (4 warps)
