@@ -39,10 +39,11 @@ L2_BYTES = 126 << 20
 # DRAM bytes per launch of the timed kernel (dram__bytes_read.sum + dram__bytes_write.sum of an ncu
 # capture), keyed by the workload string of the JSON line; None until a capture of that launch exists.
 NCU_TRAFFIC_BYTES = {
-    # measured with ncu at batch 32 (head-group kernel): 209.39 MB read + 4.44 MB written per launch;
-    # traffic grows in proportion to the batch, so a batch-256 launch moves 8 x that
+    # measured with ncu at batch 32 (head-group kernel with producer warps, the form a batch-256 launch
+    # takes): 209.39 MB read + 4.48 MB written per launch; traffic grows in proportion to the batch, so
+    # a batch-256 launch moves 8 x that
     "config5_paged_sweep B=256 Hq=32 Hkv=32 D=128 Lp=200 grid=64x64+1 paged16 sparse grid-mask window=512 n_att=208":
-        8 * 213_825_024,
+        8 * 213_865_600,
 }
 
 
