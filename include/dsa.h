@@ -234,6 +234,10 @@ DSA_API int32_t dsa_last_cuda_error(void);
  * usable (the numbers of that call are then wrong).  0 in a healthy run.  count_out: host pointer.
  * Synchronises with the device (a copy from a device symbol): not for use inside a capture. */
 DSA_API int32_t dsa_wait_timeouts(int32_t *count_out);
+/* Test hook for that mechanism: launches one warp on `stream` that waits, with the same bound, on an
+ * mbarrier nothing ever arrives on.  The wait runs out after about a second, the counter above goes
+ * up by one, the kernel ends and the context stays usable.  Asynchronous like every launch. */
+DSA_API int32_t dsa_debug_wait_giveup(void *stream);
 
 /*
  * Configure every kernel variant of the library for the CURRENT device (a few hundred one-time

@@ -39,7 +39,7 @@ EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_works
            "dsa_combine_splits", "dsa_debug_kept_indices",
            "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
            "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len", "dsa_prepare",
-           "dsa_wait_timeouts"]
+           "dsa_wait_timeouts", "dsa_debug_wait_giveup"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -103,6 +103,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_host_io.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_wait_timeouts.restype = i32
     lib.dsa_wait_timeouts.argtypes = [ctypes.POINTER(i32)]
+    lib.dsa_debug_wait_giveup.restype = i32
+    lib.dsa_debug_wait_giveup.argtypes = [vp]
     lib.dsa_prepare.restype = i32
     lib.dsa_prepare.argtypes = []
     lib.dsa_decode_step.restype = i32
@@ -252,6 +254,12 @@ def dsa_wait_timeouts() -> int:
     n = ctypes.c_int32(0)
     _check("dsa_wait_timeouts", _lib.dsa_wait_timeouts(ctypes.byref(n)))
     return int(n.value)
+
+
+def dsa_debug_wait_giveup(stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Launch the one-warp kernel whose bounded wait runs out (about a second); dsa_wait_timeouts() then
+    counts one more."""
+    _check("dsa_debug_wait_giveup", _lib.dsa_debug_wait_giveup(_stream(stream)))
 
 
 def dsa_query_plan(problem: Problem, diag: Optional[Diag] = None) -> dsa_plan_info:

@@ -775,6 +775,15 @@ const char* dsa_status_string(int32_t status) {
 
 int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
 
+int32_t dsa_debug_wait_giveup(void* stream) {
+    int* counter = nullptr;
+    const cudaError_t e0 = wait_timeouts_address(&counter);
+    if (e0 != cudaSuccess) return cuda_fail(e0);
+    dsa_wait_giveup_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(counter);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
+}
+
 int32_t dsa_wait_timeouts(int32_t* count_out) {
     if (!count_out) return DSA_ERR_INVALID_ARG;
     int n = 0;

@@ -34,27 +34,12 @@
 
 namespace dsa {
 
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// one probe of phase `parity` of the barrier (the instruction itself blocks for a bounded time)
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
-    unsigned done;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return done != 0;
-}
 // rows r.x, r.y, r.z, r.w of the view, columns [x, x + box width), to 4 consecutive box rows at dst
 __device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, int x, int4 r, unsigned long long* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes "
                  "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
                  ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w), "r"(smem_u32(bar)) : "memory");
 }
-constexpr long long kGatherWaitCycles = 1ll << 31;      // ~1 s: a wait that long gives up (see wait_timeouts)
 
 template <int D, int W, int STAGES>
 struct GatherCfg {
@@ -270,16 +255,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_gather_kernel(const AttnArgs 
         for (int tile = 0; tile < n_tiles; ++tile) {
             // Bounded wait for the tile: a copy that never lands is counted once, the kernel stops
             // waiting and runs to its end (its numbers are then wrong; dsa_wait_timeouts tells).
-            if (!gave_up) {
-                const unsigned parity = (phases >> cslot) & 1u;
-                if (!mbar_try_wait(bars + cslot, parity)) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(bars + cslot, parity)) {
-                        if (clock64() - t0 > kGatherWaitCycles) { gave_up = true; break; }
-                    }
-                    if (gave_up && lane == 0 && a.wait_timeouts) atomicAdd(a.wait_timeouts, 1);
-                }
-            }
+            mbar_wait_bounded(bars + cslot, (phases >> cslot) & 1u, gave_up, a.wait_timeouts, lane);
             phases ^= 1u << cslot;
             __syncwarp();                               // the slot consumed before this one is free for every lane
             issue_one();

@@ -33,25 +33,6 @@
 
 namespace dsa {
 
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// the barrier gets one arrival from this thread when all cp.async copies it has issued so far have landed
-__device__ __forceinline__ void cp_async_arrive_on(unsigned long long* bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Wait for phase `parity` of `bar`, for kGatherWaitCycles at most.  `gave_up` is sticky: once a wait
-// has run out the warp does not wait again.
-__device__ __forceinline__ void mbar_wait_bounded(unsigned long long* bar, unsigned parity, bool& gave_up,
-                                                  int* wait_timeouts, int lane) {
-    if (gave_up || mbar_try_wait(bar, parity)) return;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kGatherWaitCycles) { gave_up = true; break; }
-    }
-    if (gave_up && lane == 0 && wait_timeouts) atomicAdd(wait_timeouts, 1);
-}
-
 // Barrier among the consumer warps only (threads [0, N)): they build the row list while the producer
 // warps, which run on a few registers, wait for it at the block barriers.
 template <int N>

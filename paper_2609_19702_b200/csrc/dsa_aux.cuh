@@ -113,6 +113,20 @@ __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_n
 }
 
 // ---- seq_len[b] += 1 (not beyond the limit): once per decode step, after the last layer's fused step
+// One warp waits, bounded, on an mbarrier that nobody ever arrives on: the wait runs out, the warp
+// counts it and the kernel ends (what the attention kernels do when a tile never lands).
+__global__ void dsa_wait_giveup_kernel(int* wait_timeouts) {
+    __shared__ __align__(8) unsigned long long bar;
+    const int lane = threadIdx.x & 31;
+    if (lane == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    bool gave_up = false;
+    mbar_wait_bounded(&bar, 0u, gave_up, wait_timeouts, lane);
+}
+
 __global__ void dsa_advance_seq_len_kernel(int* seq_len, int batch, int limit) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < batch && seq_len[b] >= 0 && seq_len[b] < limit) seq_len[b] += 1;

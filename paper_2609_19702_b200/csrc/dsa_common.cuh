@@ -140,6 +140,42 @@ __device__ __forceinline__ void cp_async_wait_upto(int n) {
     }
 }
 
+// ---- mbarrier helpers (producer / consumer hand-over, tensor-map copies) ------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// one probe of phase `parity` of the barrier (the instruction itself blocks for a bounded time)
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+    unsigned done;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+constexpr long long kMbarWaitCycles = 1ll << 31;        // ~1 s: a wait that long gives up (see AttnArgs::wait_timeouts)
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// the barrier gets one arrival from this thread when all cp.async copies it has issued so far have landed
+__device__ __forceinline__ void cp_async_arrive_on(unsigned long long* bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Wait for phase `parity` of `bar`, for kMbarWaitCycles at most.  `gave_up` is sticky: once a wait
+// has run out the warp does not wait again.
+__device__ __forceinline__ void mbar_wait_bounded(unsigned long long* bar, unsigned parity, bool& gave_up,
+                                                  int* wait_timeouts, int lane) {
+    if (gave_up || mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kMbarWaitCycles) { gave_up = true; break; }
+    }
+    if (gave_up && lane == 0 && wait_timeouts) atomicAdd(wait_timeouts, 1);
+}
+
+
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
