@@ -14,10 +14,12 @@
  *     are HOST memory, read during the call only.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream);
  *     the library never synchronises and allocates no device memory.  It reads no environment
- *     variable and carries no result from one call to the next; what it does remember per device
- *     are idempotent set-up caches (which kernel variants have been configured, the SM count, the
- *     address of the built-in scratch array), written with atomics, so calls may come from several
- *     host threads.  Scratch comes from the caller's `workspace` (device, 256-byte aligned), sized
+ *     variable and carries no result from one call to the next (the one piece of device state that
+ *     outlives a call is a diagnostic counter, see dsa_wait_timeouts()); what it does remember per
+ *     device are idempotent set-up caches (which kernel variants have been configured, the SM
+ *     count, the addresses of the built-in scratch array and of that counter, the driver entry
+ *     point that encodes tensor maps), written with atomics, so calls may come from several host
+ *     threads.  Scratch comes from the caller's `workspace` (device, 256-byte aligned), sized
  *     by dsa_workspace_size(); it may be reused by the next call on the same stream.  The one
  *     exception is dsa_decode_attention_static_scratch(), whose scratch is a fixed array inside
  *     the library image.

@@ -802,6 +802,9 @@ int32_t dsa_prepare(void) {
     if (e == cudaSuccess) e = kernel_prepare<float, 128>();
     void* scratch = nullptr;
     if (e == cudaSuccess) e = static_scratch_address(&scratch);   // (and remember it for this device)
+    int* counter = nullptr;
+    if (e == cudaSuccess) e = wait_timeouts_address(&counter);    // (likewise: the give-up counter of the bounded waits)
+    tensor_map_encoder();                                         // (and the driver entry point the tensor-map form needs)
     sm_count();
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
