@@ -215,7 +215,7 @@ typedef struct dsa_plan_info {
     int32_t heads_per_block;/* head-group tensor-core kernel: kv heads that share the one row list */
                             /* a block builds (its warps stream heads_per_block / block_warps      */
                             /* heads each, back to back); 0: another kernel                        */
-    int32_t block_warps;    /* warps per thread block                                              */
+    int32_t block_warps;    /* warps per thread block that compute (producer_warps come on top)     */
     int32_t per_head_lists; /* 1: the per-head-list tensor-core kernel (list masks per head, fused  */
                             /* selection): shared tables per block, one candidate list per head    */
     int32_t cluster_blocks; /* blocks of a thread-block cluster that share one work item and merge */
