@@ -422,7 +422,7 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
     layers, each with its own KV cache (together larger than the L2).  Every step appends the new
     token's K/V and attends, layer after layer: one fused dsa_decode_step per layer, the layers
     sharing one seq_len array that is advanced once per token ("_two_calls" modes: dsa_append_kv +
-    attention per layer instead).  The step is captured once as a CUDA graph and replayed 1024
+    attention per layer instead); layers 2 ... n of a token carry DSA_PLAN_METADATA_STABLE.  The step is captured once as a CUDA graph and replayed 1024
     times.  Sparse: bounded ring cache, window 512, N_att 52 (95 % sparsity), grid mask.  Dense:
     full linear cache."""
     b, h, d, l_p, grid = batch, 32, 128, 50, 32
@@ -446,14 +446,19 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
         k_new, v_new = q.clone(), q.clone()
         shared_seq = torch.full((b,), l_p, dtype=torch.int32, device=dev)
         layers = []
-        for _ in range(n_layers):
+        for index in range(n_layers):
             kc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
             vc = torch.randn((b, cap, h, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
             seq = shared_seq if fused else torch.full((b,), l_p, dtype=torch.int32, device=dev)
             pl = torch.full((b,), l_p, dtype=torch.int32, device=dev)
+            # Every fused step but a token's first follows another layer's step, which writes neither the
+            # lengths nor a skip list of this layer: those calls carry the promise that lets the kernel
+            # build its row list before it waits for the launch in front of it.  (The first layer follows
+            # dsa_advance_seq_len, which writes seq_len.)
+            promise = dsa.DSA_PLAN_METADATA_STABLE if (fused and index > 0) else 0
             prob = dsa.Problem(q=q, k_cache=kc.view(-1), v_cache=vc.view(-1), strides=(cap * row, row, d),
                                seq_len=seq, prompt_len=pl, num_kv_heads=h, max_seq_len=s_max,
-                               max_prompt_len=l_p, ring_size=ring, plan_flags=plan_flags)
+                               max_prompt_len=l_p, ring_size=ring, plan_flags=plan_flags | promise)
             out, lse = dsa.alloc_outputs(prob)
             ldiag = diag
             if kind == "sparse_select":

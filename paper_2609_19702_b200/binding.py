@@ -26,6 +26,7 @@ DSA_PLAN_HEADS_PER_WARP_SHIFT = 8
 DSA_PLAN_NO_CLUSTER, DSA_PLAN_CLUSTER2, DSA_PLAN_CLUSTER4 = 0x80, 0x10000, 0x20000
 DSA_PLAN_GATHER, DSA_PLAN_NO_GATHER = 0x40000, 0x80000
 DSA_PLAN_PRODUCERS, DSA_PLAN_NO_PRODUCERS = 0x100000, 0x200000
+DSA_PLAN_METADATA_STABLE = 0x800000
 
 
 def plan_group(warps: int, heads_per_warp: int) -> int:

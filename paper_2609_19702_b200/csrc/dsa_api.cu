@@ -46,7 +46,7 @@ constexpr uint32_t kKnownPlanFlags = DSA_PLAN_CUDA_CORES | DSA_PLAN_NO_ITEM_WARP
                                      DSA_PLAN_RING_SHALLOW | DSA_PLAN_GROUP | DSA_PLAN_NO_GROUP |
                                      DSA_PLAN_GROUP_W4 | DSA_PLAN_HEADS_PER_WARP_MASK | DSA_PLAN_NO_CLUSTER |
                                      DSA_PLAN_CLUSTER2 | DSA_PLAN_CLUSTER4 | DSA_PLAN_GATHER | DSA_PLAN_NO_GATHER | DSA_PLAN_PRODUCERS |
-                                     DSA_PLAN_NO_PRODUCERS;
+                                     DSA_PLAN_NO_PRODUCERS | DSA_PLAN_METADATA_STABLE;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -563,6 +563,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->sel_val_part = nullptr; a->sel_off_part = nullptr; a->sel_k = nullptr;
     a->step_append = 0; a->k_new = nullptr; a->v_new = nullptr;
     a->wait_timeouts = nullptr;
+    a->early_list = (p->plan_flags & DSA_PLAN_METADATA_STABLE) ? 1 : 0;
 }
 
 // `after_attention`: the combine follows the attention kernel of the same call.  It is then

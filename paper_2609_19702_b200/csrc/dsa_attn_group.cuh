@@ -37,7 +37,9 @@ struct GroupCfg {
     }
 };
 
-template <int D, int G, int STAGES, int W, bool APPEND>
+// EARLY: the caller has promised that the launch before this one does not write the arrays the row
+// list is made from (AttnArgs::early_list), so the list is built before waiting for that launch.
+template <int D, int G, int STAGES, int W, bool APPEND, bool EARLY = false>
 __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a) {
     using C = GroupCfg<D, W, STAGES>;
     using IC = MmaItemCfg<D, G, false, false>;
@@ -47,7 +49,8 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
 
     // may be scheduled early behind the previous kernel of the stream, and lets the next one in early
     asm volatile("griddepcontrol.launch_dependents;");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    constexpr bool early = EARLY;
+    if constexpr (!EARLY) asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_warp[W];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -80,7 +83,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
             dst[kk][1] = hq < G ? q1 : 0u;
         }
     };
-    load_q(kvh0, qb);
+    if constexpr (!EARLY) load_q(kvh0, qb);
 
     bool has_new = false;
     const int S_step = APPEND ? step_seq_len(a, seq_raw, has_new) : seq_raw;
@@ -91,9 +94,9 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
     // reads that slot in this launch), for each of this warp's heads
     int64_t new_off = 0;
     int new_r = -1;
-    if (APPEND && has_new) {
-        new_off = token_offset(a, b, m.L_p, m.S - 1) * 2;
-        if (split == 0 && lane < 2 * C::CPR) {
+    if (APPEND && has_new) new_off = token_offset(a, b, m.L_p, m.S - 1) * 2;
+    auto store_new = [&]() {
+        if (APPEND && has_new && split == 0 && lane < 2 * C::CPR) {
             const bool is_k = lane < C::CPR;
             const int c = is_k ? lane : lane - C::CPR;
             const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_k ? a.k_new : a.v_new) + c * 16;
@@ -104,7 +107,8 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
                     *reinterpret_cast<const uint4*>(src0 + ((int64_t)b * a.H_kv + kvh) * C::ROW_BYTES);
             }
         }
-    }
+    };
+    if constexpr (!EARLY) store_new();
 
     // ---- staging --------------------------------------------------------------------------------
     // tile `tile` of head u (rows [16 tile, 16 tile + 16) of the list, of which rows_ready exist)
@@ -146,13 +150,13 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
     int i_u = 0, i_t = 0;                             // next tile to issue: head i_u, tile i_t
     {
         const int whole_a = (n_direct - (APPEND ? 1 : 0)) / MMA_KEYS;   // (never the newest row: it may not be in the cache)
-        const int early = min(STAGES - 1, max(whole_a, 0));
-        for (int s = 0; s < early; ++s) {
+        const int n_first = early ? 0 : min(STAGES - 1, max(whole_a, 0));          // (no cache reads before the wait)
+        for (int s = 0; s < n_first; ++s) {
             issue_tile(0, s, islot, n_direct);
             cp_async_commit();
             islot = islot + 1 == STAGES ? 0 : islot + 1;
         }
-        i_t = early;
+        i_t = n_first;
     }
     const int n_early = i_t;
     int n_rows = n_direct;
@@ -171,6 +175,11 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
 #pragma unroll 4
         for (int i = n_direct + (int)threadIdx.x; i < n_rows; i += NTHR)
             rowoff[i] = token_offset(a, b, m.L_p, (int)rowoff[i]) * 2;
+    }
+    if constexpr (EARLY) {                            // the list is built: now wait for the kernel before this one
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        load_q(kvh0, qb);
+        store_new();
     }
     if (n_rows <= 0) {
         for (int u = 0; u < U; ++u) write_empty_item<IC, 32>(a, m, b, kvh0 + u * W, split, lane);

@@ -47,7 +47,10 @@ struct HeadsCfg {
     }
 };
 
-template <int D, int G, int STAGES, int W, bool HEADMASK, bool SELECT, bool APPEND>
+// EARLY: the caller has promised that the launch before this one does not write the lengths, the block
+// table or the skip lists (AttnArgs::early_list): the shared tables and the first head's kept rows are
+// worked out before waiting for that launch; q, the new rows and the caches are touched after.
+template <int D, int G, int STAGES, int W, bool HEADMASK, bool SELECT, bool APPEND, bool EARLY = false>
 __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a) {
     using C = HeadsCfg<D, G, STAGES, W, HEADMASK>;
     using T = __nv_bfloat16;
@@ -56,7 +59,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
     constexpr int NTHR = 32 * W;
 
     asm volatile("griddepcontrol.launch_dependents;");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if constexpr (!EARLY) asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ __align__(128) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char* ring = smem + warp * (STAGES * C::SLOT_BYTES);
@@ -93,7 +96,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
             dst[kk][1] = hq < G ? q1 : 0u;
         }
     };
-    load_q(kvh0, qb);
+    if constexpr (!EARLY) load_q(kvh0, qb);
 
     bool has_new = false;
     const int S_step = APPEND ? step_seq_len(a, seq_raw, has_new) : seq_raw;
@@ -104,18 +107,21 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
     const int r_lo = split * a.chunk;                 // ranks [r_lo, r_lo + chunk) of the kept sequence are this split's rows
 
     // fused step: the token being decoded goes from k_new / v_new to the cache (split 0), per head
-    if (APPEND && has_new && split == 0 && lane < 2 * C::CPR) {
-        const int64_t new_off = token_offset(a, b, m.L_p, m.S - 1) * 2;
-        const bool is_k = lane < C::CPR;
-        const int c = is_k ? lane : lane - C::CPR;
-        const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_k ? a.k_new : a.v_new) + c * 16;
-        unsigned char* dst0 = const_cast<unsigned char*>(is_k ? kbase : vbase) + new_off + c * 16;
-        for (int u = 0; u < U; ++u) {
-            const int kvh = kvh0 + u * W;
-            *reinterpret_cast<uint4*>(dst0 + kvh * head_stride_bytes) =
-                *reinterpret_cast<const uint4*>(src0 + ((int64_t)b * a.H_kv + kvh) * C::ROW_BYTES);
+    auto store_new = [&]() {
+        if (APPEND && has_new && split == 0 && lane < 2 * C::CPR) {
+            const int64_t new_off = token_offset(a, b, m.L_p, m.S - 1) * 2;
+            const bool is_k = lane < C::CPR;
+            const int c = is_k ? lane : lane - C::CPR;
+            const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_k ? a.k_new : a.v_new) + c * 16;
+            unsigned char* dst0 = const_cast<unsigned char*>(is_k ? kbase : vbase) + new_off + c * 16;
+            for (int u = 0; u < U; ++u) {
+                const int kvh = kvh0 + u * W;
+                *reinterpret_cast<uint4*>(dst0 + kvh * head_stride_bytes) =
+                    *reinterpret_cast<const uint4*>(src0 + ((int64_t)b * a.H_kv + kvh) * C::ROW_BYTES);
+            }
         }
-    }
+    };
+    if constexpr (!EARLY) store_new();
 
     // ---- shared by all heads of the block: where the always-kept rows and the window candidates live
     for (int r = threadIdx.x; r < prefix; r += NTHR)
@@ -260,7 +266,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
     int n_early = 0;
     {
         const int whole = dir_rows / MMA_KEYS;
-        n_early = min(STAGES - 1, whole);
+        n_early = EARLY ? 0 : min(STAGES - 1, whole);       // (no cache reads before the wait)
         for (int s = 0; s < n_early; ++s) {
             issue_tile(kvh0, s, islot, dir_rows, -1);
             cp_async_commit();
@@ -295,6 +301,11 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
     int cur_kept = build_kidx(kvh0, 0, pre);
     if (U > 1) prefetch_trace(kvh0 + W, pre);
     convert(0, cur_kept);
+    if constexpr (EARLY) {                            // the first head's rows are known: now wait for the kernel before this one
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        load_q(kvh0, qb);
+        store_new();
+    }
     int cur_rows = rows_of(cur_kept);
     int cur_new = new_row_of(0, cur_kept, cur_rows);
     int cur_tiles = (cur_rows + MMA_KEYS - 1) / MMA_KEYS;

@@ -133,11 +133,17 @@ struct KernelPick {
             return w == 4 ? smem_group_w<4, kGroupStagesShallow>(chunk, bw) : smem_group_w<2, kGroupStagesShallow>(chunk, bw);
         return w == 4 ? smem_group_w<4, kGroupStages>(chunk, bw) : smem_group_w<2, kGroupStages>(chunk, bw);
     }
-    template <int W, bool APPEND, int ST>
+    template <int W, bool APPEND, int ST, bool EARLY = false>
     static ConfiguredFlags* group_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
     template <int W, bool APPEND, int ST>
     static cudaError_t launch_group_w(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
         if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            if (W == 4 && a.early_list) {               // (the early-list form exists for four-warp blocks)
+                auto kern = dsa_attn_group_kernel<D, G, ST, 4, APPEND, true>;
+                const cudaError_t e = ensure_configured(kern, group_configured<4, APPEND, ST, true>());
+                if (e != cudaSuccess) return e;
+                return launch_pdl(kern, (unsigned)blocks, 32 * 4, smem_bytes, st, a);
+            }
             auto kern = dsa_attn_group_kernel<D, G, ST, W, APPEND>;
             const cudaError_t e = ensure_configured(kern, group_configured<W, APPEND, ST>());
             if (e != cudaSuccess) return e;
@@ -214,11 +220,17 @@ struct KernelPick {
     static size_t smem_heads(int dir_cap, int window, int kidx_cap, int bw) {
         return HeadsCfg<D, G, kMmaStages, kHeadsWarps, HM>::smem_bytes(dir_cap, window, kidx_cap, bw);
     }
-    template <bool APPEND>
+    template <bool APPEND, bool EARLY = false>
     static ConfiguredFlags* heads_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
     template <bool APPEND>
     static cudaError_t launch_heads_a(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
+            if (a.early_list) {
+                auto kern = dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, APPEND, true>;
+                const cudaError_t e = ensure_configured(kern, heads_configured<APPEND, true>());
+                if (e != cudaSuccess) return e;
+                return launch_pdl(kern, (unsigned)blocks, 32 * kHeadsWarps, smem_bytes, st, a);
+            }
             auto kern = dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, APPEND>;
             const cudaError_t e = ensure_configured(kern, heads_configured<APPEND>());
             if (e != cudaSuccess) return e;
@@ -245,6 +257,10 @@ struct KernelPick {
                 e = ensure_configured(dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, false>, heads_configured<false>());
             if (e == cudaSuccess)
                 e = ensure_configured(dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, true>, heads_configured<true>());
+            if (e == cudaSuccess)
+                e = ensure_configured(dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, false, true>, heads_configured<false, true>());
+            if (e == cudaSuccess)
+                e = ensure_configured(dsa_attn_heads_kernel<D, G, kMmaStages, kHeadsWarps, HM, SEL, true, true>, heads_configured<true, true>());
             using one = std::integral_constant<int, 1>;
             using two = std::integral_constant<int, 2>;
             using four = std::integral_constant<int, kMmaItemWarps>;
@@ -271,6 +287,11 @@ struct KernelPick {
                     constexpr bool APPEND = decltype(app)::value;
                     if (e == cudaSuccess)
                         e = ensure_configured(dsa_attn_group_kernel<D, G, ST, W, APPEND>, group_configured<W, APPEND, ST>());
+                    if constexpr (W == 4) {
+                        if (e == cudaSuccess)
+                            e = ensure_configured(dsa_attn_group_kernel<D, G, ST, 4, APPEND, true>,
+                                                  group_configured<4, APPEND, ST, true>());
+                    }
                 };
                 using gdeep = std::integral_constant<int, kGroupStages>;
                 using gshallow = std::integral_constant<int, kGroupStagesShallow>;
