@@ -145,8 +145,9 @@ typedef struct dsa_problem {
 #define DSA_PLAN_NO_PRODUCERS  0x200000u /* never                                                       */
 /* Not a planner switch but a promise about the stream: the launch just before this call does not write
  * seq_len, prompt_len, block_table or the skip lists (in a model it is the projection that produces q
- * and the new K / V rows).  Kernels that chain with programmatic dependent launch then work out which
- * rows to read BEFORE they wait for that launch and touch q, the new rows and the caches only after. */
+ * and the new K / V rows, or the previous layer's attention).  The head-group and per-head-list kernels,
+ * which chain with programmatic dependent launch, then work out which rows to read BEFORE they wait
+ * for that launch, and touch q, the new rows and the caches only after; other kernels ignore it. */
 #define DSA_PLAN_METADATA_STABLE 0x800000u
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u
