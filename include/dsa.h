@@ -143,11 +143,15 @@ typedef struct dsa_problem {
 #define DSA_PLAN_NO_GATHER     0x80000u /* never do                                                        */
 #define DSA_PLAN_PRODUCERS     0x100000u /* head-group kernel, 4 warps: a producer warp beside every consumer warp */
 #define DSA_PLAN_NO_PRODUCERS  0x200000u /* never                                                       */
-/* Not a planner switch but a promise about the stream: the launch just before this call does not write
- * seq_len, prompt_len, block_table or the skip lists (in a model it is the projection that produces q
- * and the new K / V rows, or the previous layer's attention).  The head-group and per-head-list kernels,
- * which chain with programmatic dependent launch, then work out which rows to read BEFORE they wait
- * for that launch, and touch q, the new rows and the caches only after; other kernels ignore it. */
+/* Not a planner switch but a promise about the stream: no launch that can still be running when this
+ * call's kernel starts writes seq_len, prompt_len, block_table or the skip lists.  The attention kernels
+ * chain with programmatic dependent launch and let their successor start before they have waited for
+ * their own predecessor, so "still running" means: the launch just before this call and, if that is an
+ * attention call of this library, the launches before it in turn, back to the first launch that is not
+ * (a projection, dsa_advance_seq_len, dsa_append_kv: those complete before anything behind them starts).
+ * In a decode loop every layer's call but the one that follows dsa_advance_seq_len can make the promise.
+ * The head-group and per-head-list kernels then work out which rows to read BEFORE they wait for the
+ * launch in front, and touch q, the new rows and the caches only after; other kernels ignore it. */
 #define DSA_PLAN_METADATA_STABLE 0x800000u
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u

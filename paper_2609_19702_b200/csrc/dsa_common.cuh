@@ -50,10 +50,10 @@ struct AttnArgs {
     const void* k_new;           // [B, H_kv, D] rows of the current token; NULL: already in the cache
     const void* v_new;
     int* wait_timeouts;          // device counter of bounded mbarrier waits that gave up (0 in a healthy run); may be NULL
-    int early_list;              // 1: the caller promises that the launch just before this one on the stream does not write
+    int early_list;              // 1: the caller promises that no launch still running when this kernel starts writes
                                  // seq_len, prompt_len, block_table or the skip lists, so the row list may be built BEFORE
-                                 // waiting for that launch (programmatic dependent launch); q, the new rows and the caches
-                                 // are still read after the wait only
+                                 // waiting for the launch in front (programmatic dependent launch); q, the new rows and
+                                 // the caches are still read after the wait only
 };
 
 // What the tensor-map (gather) kernel needs beyond AttnArgs: the K and V caches as 2-D views
