@@ -147,9 +147,11 @@ typedef struct dsa_problem {
  * call's kernel starts writes seq_len, prompt_len, block_table or the skip lists.  The attention kernels
  * chain with programmatic dependent launch and let their successor start before they have waited for
  * their own predecessor, so "still running" means: the launch just before this call and, if that is an
- * attention call of this library, the launches before it in turn, back to the first launch that is not
- * (a projection, dsa_advance_seq_len, dsa_append_kv: those complete before anything behind them starts).
- * In a decode loop every layer's call but the one that follows dsa_advance_seq_len can make the promise.
+ * attention call of this library, the launches before it in turn, back to the first launch that does
+ * not let its successor in early (a projection, dsa_advance_seq_len: those complete before anything
+ * behind them starts).  dsa_append_kv does let its successor in early and, when it advances, writes
+ * seq_len: the call behind it cannot make the promise.  In a decode loop of fused steps every layer's
+ * call but the one that follows dsa_advance_seq_len can.
  * The head-group and per-head-list kernels then work out which rows to read BEFORE they wait for the
  * launch in front, and touch q, the new rows and the caches only after; other kernels ignore it. */
 #define DSA_PLAN_METADATA_STABLE 0x800000u

@@ -112,7 +112,6 @@ __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_n
     if (advance && threadIdx.x == 0) a.seq_len_rw[b] = S + 1;
 }
 
-// ---- seq_len[b] += 1 (not beyond the limit): once per decode step, after the last layer's fused step
 // One warp waits, bounded, on an mbarrier that nobody ever arrives on: the wait runs out, the warp
 // counts it and the kernel ends (what the attention kernels do when a tile never lands).
 __global__ void dsa_wait_giveup_kernel(int* wait_timeouts) {
@@ -127,6 +126,8 @@ __global__ void dsa_wait_giveup_kernel(int* wait_timeouts) {
     mbar_wait_bounded(&bar, 0u, gave_up, wait_timeouts, lane);
 }
 
+// ---- seq_len[b] += 1 (not beyond the limit): once per decode step, after the last layer's fused step.
+// A plain launch that does not signal early: everything queued behind it sees the new lengths.
 __global__ void dsa_advance_seq_len_kernel(int* seq_len, int batch, int limit) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < batch && seq_len[b] >= 0 && seq_len[b] < limit) seq_len[b] += 1;
