@@ -152,8 +152,9 @@ typedef struct dsa_problem {
  * behind them starts).  dsa_append_kv does let its successor in early and, when it advances, writes
  * seq_len: the call behind it cannot make the promise.  In a decode loop of fused steps every layer's
  * call but the one that follows dsa_advance_seq_len can.
- * The head-group and per-head-list kernels then work out which rows to read BEFORE they wait for the
- * launch in front, and touch q, the new rows and the caches only after; other kernels ignore it. */
+ * The head-group, per-head-list, several-warps-per-item and cluster kernels then work out which rows to
+ * read BEFORE they wait for the launch in front, and touch q, the new rows and the caches only after;
+ * the other kernels (producer-warp and tensor-map forms, one warp per item, CUDA cores) ignore it. */
 #define DSA_PLAN_METADATA_STABLE 0x800000u
 #define DSA_PLAN_HEADS_PER_WARP_SHIFT 8  /* forced head-group kernel: kv heads per warp in bits 8..15    */
 #define DSA_PLAN_HEADS_PER_WARP_MASK  0xff00u

@@ -118,7 +118,11 @@ struct MmaItemCfg {
 // block 0 then reads the other blocks' merged states straight out of their shared memory
 // (ld.shared::cluster after a cluster barrier) and writes the result: no partials in HBM, no combine
 // launch.  The launch carries the cluster dimension; plain per-thread loads only cross the cluster.
-template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false, int KW = 1, int CL = 1>
+// EARLY: the caller has promised that no launch still running writes the arrays the row list is made
+// from (AttnArgs::early_list): the list is built before waiting for the launch in front; q, the new rows
+// and the caches are read after the wait.
+template <int D, int G, int STAGES, bool HEADMASK, bool SELECT, int W, bool APPEND = false, int KW = 1, int CL = 1,
+          bool EARLY = false>
 __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArgs a) {
     using C = MmaCfg<D, G, STAGES, HEADMASK, SELECT, W * KW>;   // one ring per warp
     using IC = MmaItemCfg<D, G, HEADMASK, SELECT>;
@@ -134,7 +138,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     // itself have been scheduled early behind the append kernel of the same decode step: wait for
     // that kernel's writes (the new K/V rows, seq_len) before touching global memory.
     asm volatile("griddepcontrol.launch_dependents;");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if constexpr (!EARLY) asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_warp[NW];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -161,7 +165,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     const int hq = lane >> 2;                 // head column this thread feeds
     const int qd = (lane & 3) * 2;
     unsigned qb[C::KSTEPS][2];
-    {
+    if constexpr (!EARLY) {
         const T* qrow = reinterpret_cast<const T*>(a.q) + ((int64_t)b * a.H_q + kvh * G + (hq < G ? hq : 0)) * D;
 #pragma unroll
         for (int kk = 0; kk < C::KSTEPS; ++kk) {
@@ -190,9 +194,11 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
         knew_row = reinterpret_cast<const unsigned char*>(a.k_new) + row_bytes;
         vnew_row = reinterpret_cast<const unsigned char*>(a.v_new) + row_bytes;
         off_new = token_offset(a, b, m.L_p, m.S - 1);
-        if (store_new) {                                  // lanes [0, CPR): K chunks, [CPR, 2 CPR): V chunks
-            const unsigned char* src = lane < C::CPR ? knew_row + lane * 16 : vnew_row + (lane - C::CPR) * 16;
-            new_chunk = *reinterpret_cast<const uint4*>(src);
+        if constexpr (!EARLY) {
+            if (store_new) {                              // lanes [0, CPR): K chunks, [CPR, 2 CPR): V chunks
+                const unsigned char* src = lane < C::CPR ? knew_row + lane * 16 : vnew_row + (lane - C::CPR) * 16;
+                new_chunk = *reinterpret_cast<const uint4*>(src);
+            }
         }
     }
 
@@ -232,11 +238,24 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
     // whole tiles inside phase A (fused step: never the newest row, which may not be in the cache)
     // that are this warp's
     const int whole_a = (n_direct - (APPEND ? 1 : 0)) / MMA_KEYS;
-    const int early = min(STAGES - 1, whole_a > wk ? (whole_a - wk + KW - 1) / KW : 0);
+    const int early = EARLY ? 0 : min(STAGES - 1, whole_a > wk ? (whole_a - wk + KW - 1) / KW : 0);   // (EARLY: no cache reads yet)
     for (int s = 0; s < early; ++s) issue_tile(s, n_direct);
     const int n_rows = NW == 1
         ? build_rows_scanned<IC, WarpSync, 32>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct)
         : build_rows_scanned<IC, BlockSync, 32 * NW>(a, m, b, list_kvh, split, list, bitmaps, s_warp, n_direct);
+    if constexpr (EARLY) {                             // the list is built: now wait for the launch in front
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const T* qrow = reinterpret_cast<const T*>(a.q) + ((int64_t)b * a.H_q + kvh * G + (hq < G ? hq : 0)) * D;
+#pragma unroll
+        for (int kk = 0; kk < C::KSTEPS; ++kk) {
+            qb[kk][0] = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd);
+            qb[kk][1] = *reinterpret_cast<const unsigned*>(qrow + kk * 16 + qd + 8);
+        }
+        if (store_new) {
+            const unsigned char* src = lane < C::CPR ? knew_row + lane * 16 : vnew_row + (lane - C::CPR) * 16;
+            new_chunk = *reinterpret_cast<const uint4*>(src);
+        }
+    }
     if (store_new) {
         unsigned char* base = const_cast<unsigned char*>(lane < C::CPR ? kbase : vbase);
         const int c = lane < C::CPR ? lane : lane - C::CPR;

@@ -96,12 +96,20 @@ struct KernelPick {
     }
     template <int W, bool APPEND, int KW, int ST>
     static ConfiguredFlags* mma_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
-    template <bool APPEND, int CL>
+    template <bool APPEND, int CL, bool EARLY = false>
     static ConfiguredFlags* cluster_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
+    template <bool APPEND>
+    static ConfiguredFlags* kw_early_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
     // several warps per item, CL blocks of a cluster per item (head-independent masks only)
     template <bool APPEND, int CL>
     static cudaError_t launch_cluster_c(const AttnArgs& a, int64_t items, size_t smem_bytes, cudaStream_t st) {
         if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            if (a.early_list) {                         // (row list before the dependency wait)
+                auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, CL, true>;
+                const cudaError_t e = ensure_configured(kern, cluster_configured<APPEND, CL, true>());
+                if (e != cudaSuccess) return e;
+                return launch_pdl_cluster(kern, (unsigned)(items * CL), 32 * kMmaItemWarps, smem_bytes, st, CL, a);
+            }
             auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, CL>;
             const cudaError_t e = ensure_configured(kern, cluster_configured<APPEND, CL>());
             if (e != cudaSuccess) return e;
@@ -270,6 +278,12 @@ struct KernelPick {
             mma(one{}, std::true_type{}, one{}, deep{});
             mma(one{}, std::false_type{}, four{}, deep{});
             mma(one{}, std::true_type{}, four{}, deep{});
+            if (e == cudaSuccess)
+                e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, false, kMmaItemWarps, 1, true>,
+                                      kw_early_configured<false>());
+            if (e == cudaSuccess)
+                e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, true, kMmaItemWarps, 1, true>,
+                                      kw_early_configured<true>());
             if constexpr (!HM && !SEL) {
                 auto cluster = [&](auto app, auto cl) {
                     constexpr bool APPEND = decltype(app)::value;
@@ -278,6 +292,17 @@ struct KernelPick {
                         e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, CL>,
                                               cluster_configured<APPEND, CL>());
                 };
+                auto cluster_early = [&](auto app, auto cl) {
+                    constexpr bool APPEND = decltype(app)::value;
+                    constexpr int CL = decltype(cl)::value;
+                    if (e == cudaSuccess)
+                        e = ensure_configured(dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, CL, true>,
+                                              cluster_configured<APPEND, CL, true>());
+                };
+                cluster_early(std::false_type{}, two{});
+                cluster_early(std::true_type{}, two{});
+                cluster_early(std::false_type{}, four{});
+                cluster_early(std::true_type{}, four{});
                 cluster(std::false_type{}, two{});
                 cluster(std::true_type{}, two{});
                 cluster(std::false_type{}, four{});
@@ -336,6 +361,12 @@ struct KernelPick {
     static cudaError_t launch_mma_a(int w, int kw, int stages, const AttnArgs& a, int64_t items, size_t smem_bytes,
                                     cudaStream_t st) {
         if constexpr (sizeof(T) == 2) {
+            if (kw > 1 && a.early_list) {               // (row list before the dependency wait)
+                auto kern = dsa_attn_mma_kernel<D, G, kMmaStages, HM, SEL, 1, APPEND, kMmaItemWarps, 1, true>;
+                const cudaError_t e = ensure_configured(kern, kw_early_configured<APPEND>());
+                if (e != cudaSuccess) return e;
+                return launch_pdl(kern, (unsigned)items, 32 * kMmaItemWarps, smem_bytes, st, a);
+            }
             if (kw > 1) return launch_mma_w<1, APPEND, kMmaItemWarps>(a, items, smem_bytes, st);
             if constexpr (!HM && !SEL) {
                 if (w == 2 && stages == kMmaStagesShallow)

@@ -1,6 +1,6 @@
 """DSA_PLAN_METADATA_STABLE: the caller's promise that the launch before a call does not write the
-lengths, the block table or the skip lists, which lets the head-group and per-head-list kernels work
-out their rows BEFORE they wait for that launch.
+lengths, the block table or the skip lists, which lets the head-group, per-head-list, several-warps-
+per-item and cluster kernels work out their rows BEFORE they wait for that launch.
 
 Two things are checked.  (1) The early-list kernels compute the same as the others: the cases of the
 other parity modules run with the promise set on every problem (and, so that it is kept whatever a
@@ -32,11 +32,12 @@ def dsa():
     return binding
 
 
-@pytest.fixture(params=[1, 2], ids=["u1", "u2"])
+@pytest.fixture(params=[1, 2, 0], ids=["u1", "u2", "planned"])
 def promised(request, dsa, monkeypatch):
-    """Every problem carries the promise (and the four-warp multi-head kernels that honour it); the
-    device is idle when a call is made."""
-    flags = dsa.plan_group(4, request.param) | dsa.DSA_PLAN_METADATA_STABLE
+    """Every problem carries the promise, with the four-warp multi-head kernels forced (1 or 2 heads per
+    warp) or with the library's own plan (the small cases then take the several-warps-per-item and
+    cluster kernels, which honour it as well); the device is idle when a call is made."""
+    flags = dsa.DSA_PLAN_METADATA_STABLE | (dsa.plan_group(4, request.param) if request.param else 0)
     orig = dsa.Problem.c_struct
 
     def patched(self):
