@@ -3,6 +3,8 @@ batch and compare.  Tolerances are the ones the task states: kept positions bit-
 |gpu - ref| <= 1e-2 + 1e-2 |ref| for bf16 outputs, |lse_gpu - lse_ref| <= 1e-3."""
 from __future__ import annotations
 
+import zlib
+
 import numpy as np
 
 from oracle import oracle as ora
@@ -13,8 +15,31 @@ OUT_ATOL, OUT_RTOL, LSE_ATOL = 1e-2, 1e-2, 1e-3
 F32_ATOL, F32_RTOL, F32_LSE_ATOL = 1e-5, 1e-5, 1e-5
 
 
+_ORACLE_MEMO = {}
+
+
+def _crc(x):
+    return None if x is None else (x.shape, str(x.dtype), zlib.crc32(np.ascontiguousarray(x).view(np.uint8).reshape(-1)))
+
+
 def oracle_run(inp, mode, *, n_r=0, n_att=0, stride=0, trace=None, n_sink=0, want_kept=False, requests=None):
-    """Oracle on a host batch (optionally on a subset of requests)."""
+    """Oracle on a host batch (optionally on a subset of requests).  Several modules run the same
+    cases under different kernel plans, so results are kept per process, keyed by checksums of every
+    input array and by the arguments (the oracle itself is untouched)."""
+    w = inp["workload"]
+    key = (mode, n_r, n_att, stride, n_sink, want_kept, None if requests is None else tuple(int(r) for r in requests),
+           w.num_kv_heads, tuple(inp["strides"]), inp["block_size"], _crc(trace),
+           tuple(_crc(inp[k]) for k in ("q", "k_cache", "v_cache", "seq_len", "prompt_len", "block_table")))
+    if key in _ORACLE_MEMO:
+        return _ORACLE_MEMO[key]
+    ref = _oracle_run(inp, mode, n_r=n_r, n_att=n_att, stride=stride, trace=trace, n_sink=n_sink, want_kept=want_kept,
+                      requests=requests)
+    if len(_ORACLE_MEMO) < 4096:
+        _ORACLE_MEMO[key] = ref
+    return ref
+
+
+def _oracle_run(inp, mode, *, n_r=0, n_att=0, stride=0, trace=None, n_sink=0, want_kept=False, requests=None):
     w = inp["workload"]
     q, seq, pl, bt = inp["q"], inp["seq_len"], inp["prompt_len"], inp["block_table"]
     if requests is not None:
