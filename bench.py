@@ -635,6 +635,29 @@ def run_ours(args):
                 "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                 "kernel": kernel_name(plan) + (" + dsa_combine_kernel" if plan.launches > 1 else "")}
 
+    # ---- the launch's own speed of light: the same call with the arithmetic taken out (same grid, same
+    # row lists, same K / V tiles staged through the same rings; dsa_debug_copy_only), timed in regions
+    # that alternate with regions of the real call so that clock drift hits both alike
+    if plan.block_warps == 4 and not plan.per_head_lists and not flush_l2 and world == 1:
+        ws_copy = dsa.alloc_workspace(prob, diag)
+
+        def copy_call():
+            dsa.dsa_debug_copy_only(prob, diag, out, lse, ws_copy)
+
+        real_t, copy_t = [], []
+        time_calls(torch, copy_call, args.steps, 3, None, barrier)
+        for _ in range(5):
+            real_t.append(time_calls(torch, call, args.steps, 0, None, barrier)[0])
+            copy_t.append(time_calls(torch, copy_call, args.steps, 0, None, barrier)[0])
+        c_secs, r_secs = float(np.median(copy_t)) / args.steps, float(np.median(real_t)) / args.steps
+        roofline["copy_only"] = {"ms_per_launch": round(c_secs * 1e3, 5), "GBs": round(abytes / c_secs / 1e9, 1),
+                                 "attention_ms_in_the_same_regions": round(r_secs * 1e3, 5),
+                                 "attention_over_copy_only": round(r_secs / c_secs, 4),
+                                 "note": "the same launch without the arithmetic (plain four-warp head-group "
+                                         "kernel with the plan's grid): lists built, tiles staged and read once"}
+        call()                                              # (out / lse hold the attention result again)
+        torch.cuda.synchronize()
+
     # ---- the same step as a single call with a cold L2 (launch latency and first misses included)
     iso_flush = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
     iso_med, iso_min = time_flushed(torch, call, iso_flush, iters=30, warmup=3)

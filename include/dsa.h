@@ -249,6 +249,14 @@ DSA_API int32_t dsa_last_cuda_error(void);
  * usable (the numbers of that call are then wrong).  0 in a healthy run.  count_out: host pointer.
  * Synchronises with the device (a copy from a device symbol): not for use inside a capture. */
 DSA_API int32_t dsa_wait_timeouts(int32_t *count_out);
+/* Measuring hook: the sparse / dense call (diag NULL: dense) with the arithmetic taken out.  The launch
+ * has the plan's grid, builds the same row lists and stages the same K / V tiles through the same
+ * shared-memory rings, but a landed tile is only read once; what it leaves in out / lse (and the
+ * workspace) is meaningless.  Its time is what the staging alone costs for this very problem -- the
+ * attention call's own speed of light.  DSA_ERR_UNSUPPORTED unless the plan is the four-warp head-group
+ * kernel (dsa_plan_info.block_warps == 4, per_head_lists == 0).  Arguments as dsa_decode_attention_sparse. */
+DSA_API int32_t dsa_debug_copy_only(const dsa_problem *problem, const dsa_diag_params *diag, void *out, float *lse,
+                                    void *workspace, size_t workspace_bytes, void *stream);
 /* Test hook for that mechanism: launches one warp on `stream` that waits, with the same bound, on an
  * mbarrier nothing ever arrives on.  The wait runs out after about a second, the counter above goes
  * up by one, the kernel ends and the context stays usable.  Asynchronous like every launch. */

@@ -40,7 +40,7 @@ EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_works
            "dsa_combine_splits", "dsa_debug_kept_indices",
            "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
            "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len", "dsa_prepare",
-           "dsa_wait_timeouts", "dsa_debug_wait_giveup"]
+           "dsa_wait_timeouts", "dsa_debug_wait_giveup", "dsa_debug_copy_only"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -104,6 +104,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_decode_attention_host_io.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_wait_timeouts.restype = i32
     lib.dsa_wait_timeouts.argtypes = [ctypes.POINTER(i32)]
+    lib.dsa_debug_copy_only.restype = i32
+    lib.dsa_debug_copy_only.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.dsa_debug_wait_giveup.restype = i32
     lib.dsa_debug_wait_giveup.argtypes = [vp]
     lib.dsa_prepare.restype = i32
@@ -304,6 +306,20 @@ def dsa_decode_attention_sparse(problem: Problem, diag: Diag, out: torch.Tensor,
     _check("dsa_decode_attention_sparse",
            _lib.dsa_decode_attention_sparse(_ref(p), _ref(d), _dptr(out), _dptr(lse), _dptr(workspace),
                                             ws_n, _stream(stream)))
+
+
+def dsa_debug_copy_only(problem: Problem, diag: Optional[Diag], out: torch.Tensor, lse: torch.Tensor,
+                        workspace: Optional[torch.Tensor] = None,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """The attention call with the arithmetic taken out (same grid, lists and K / V staging; out and lse
+    come back meaningless): what the staging alone costs.  Raises DsaError (unsupported) unless the plan
+    is the four-warp head-group kernel."""
+    p = problem.c_struct()
+    d = diag.c_struct() if diag is not None else None
+    ws_n = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check("dsa_debug_copy_only",
+           _lib.dsa_debug_copy_only(_ref(p), _ref(d), _dptr(out), _dptr(lse), _dptr(workspace), ws_n,
+                                    _stream(stream)))
 
 
 def dsa_decode_attention_static_scratch(problem: Problem, diag: Optional[Diag], out: torch.Tensor,

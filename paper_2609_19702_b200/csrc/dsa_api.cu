@@ -71,6 +71,7 @@ struct Plan {
     int group_u;         // and kv heads each warp streams through the block's one row list
     int group_stages;    // and its ring depth
     bool producers;      // and whether every ring has a producer warp beside its consumer warp
+    bool copy_only;      // measuring form of the plain four-warp kernel (dsa_debug_copy_only)
     bool gather;         // and whether its tiles are staged by tensor-map gather copies; the 2-D cache view then:
     int gather_rows_per_stride_b;
     int64_t gather_rows; // its number of token rows
@@ -101,7 +102,7 @@ KernelQuery kernel_query(const Plan& pl) {
     q.G = pl.G; q.headmask = pl.headmask; q.select = pl.select;
     q.mma = pl.mma; q.mma_warps = pl.mma_warps; q.mma_kw = pl.mma_kw; q.mma_stages = pl.mma_stages;
     q.mma_cl = pl.mma_cl;
-    q.group_w = pl.group_w; q.group_stages = pl.group_stages; q.gather = pl.gather; q.producers = pl.producers;
+    q.group_w = pl.group_w; q.group_stages = pl.group_stages; q.gather = pl.gather; q.producers = pl.producers; q.copy_only = pl.copy_only;
     q.heads = pl.heads; q.dir_cap = pl.dir_cap; q.kidx_cap = pl.kidx_cap; q.window = pl.window;
     return q;
 }
@@ -276,6 +277,7 @@ int32_t make_plan(const dsa_problem* p, const dsa_diag_params* d, Plan* pl) {
     pl->group_stages = kGroupStages;
     pl->gather = false;
     pl->producers = false;
+    pl->copy_only = false;
     pl->gather_rows_per_stride_b = 0;
     pl->gather_rows = 0;
     pl->heads = false;
@@ -674,10 +676,17 @@ int32_t build_gather_maps(const dsa_problem* p, const Plan& pl, GatherMaps* g) {
 // token being decoded is appended by this call and attended to as well.
 int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out, float* lse,
                       void* workspace, size_t workspace_bytes, void* stream, const void* k_new = nullptr,
-                      const void* v_new = nullptr) {
+                      const void* v_new = nullptr, bool copy_only = false) {
     Plan pl;
     int32_t rc = make_plan(p, d, &pl);
     if (rc != DSA_OK) return rc;
+    if (copy_only) {
+        // the measuring form exists for the plain four-warp head-group kernel: same grid, same lists, same copies
+        if (pl.group_w != 4 || pl.heads || k_new) return DSA_ERR_UNSUPPORTED;
+        pl.producers = false;
+        pl.gather = false;
+        pl.copy_only = true;
+    }
     if (p->batch == 0) return DSA_OK;
     if (!out || !lse || !aligned16(out)) return DSA_ERR_INVALID_ARG;
     const bool step = k_new != nullptr;
@@ -775,6 +784,11 @@ const char* dsa_status_string(int32_t status) {
 }
 
 int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
+
+int32_t dsa_debug_copy_only(const dsa_problem* problem, const dsa_diag_params* diag, void* out, float* lse,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    return run_attention(problem, diag, out, lse, workspace, workspace_bytes, stream, nullptr, nullptr, true);
+}
 
 int32_t dsa_debug_wait_giveup(void* stream) {
     int* counter = nullptr;

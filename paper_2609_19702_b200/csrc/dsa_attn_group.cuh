@@ -39,7 +39,10 @@ struct GroupCfg {
 
 // EARLY: the caller has promised that the launch before this one does not write the arrays the row
 // list is made from (AttnArgs::early_list), so the list is built before waiting for that launch.
-template <int D, int G, int STAGES, int W, bool APPEND, bool EARLY = false>
+// COPY_ONLY: a measuring form (dsa_debug_copy_only): the same lists, the same copies into the same rings,
+// but a landed tile is only read once and folded, no arithmetic; what it writes to out / lse is meaningless.
+// Its time is what this launch's staging alone costs: the kernel's own speed of light.
+template <int D, int G, int STAGES, int W, bool APPEND, bool EARLY = false, bool COPY_ONLY = false>
 __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a) {
     using C = GroupCfg<D, W, STAGES>;
     using IC = MmaItemCfg<D, G, false, false>;
@@ -225,6 +228,17 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_group_kernel(const AttnArgs a
             const unsigned char* ks = ring + cslot * C::SLOT_BYTES;
             const unsigned char* vs = ks + C::TILE_BYTES;
             cslot = cslot + 1 == STAGES ? 0 : cslot + 1;
+            if constexpr (COPY_ONLY) {
+                const uint4* p = reinterpret_cast<const uint4*>(ks);
+                uint4 f = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int i = 0; i < C::SLOT_BYTES / 512; ++i) {
+                    const uint4 x = p[i * 32 + lane];
+                    f.x ^= x.x; f.y ^= x.y; f.z ^= x.z; f.w ^= x.w;
+                }
+                lpart[0] += __uint_as_float((f.x ^ f.y ^ f.z ^ f.w) & 0x007fffffu);    // (kept alive; tiny and finite)
+                continue;
+            }
 
             // S^T = K . Q^T
             float s[4] = {0.f, 0.f, 0.f, 0.f};

@@ -141,11 +141,20 @@ struct KernelPick {
             return w == 4 ? smem_group_w<4, kGroupStagesShallow>(chunk, bw) : smem_group_w<2, kGroupStagesShallow>(chunk, bw);
         return w == 4 ? smem_group_w<4, kGroupStages>(chunk, bw) : smem_group_w<2, kGroupStages>(chunk, bw);
     }
-    template <int W, bool APPEND, int ST, bool EARLY = false>
+    template <int W, bool APPEND, int ST, bool EARLY = false, bool COPY_ONLY = false>
     static ConfiguredFlags* group_configured() { static ConfiguredFlags done[kMaxDevices] = {}; return done; }
     template <int W, bool APPEND, int ST>
-    static cudaError_t launch_group_w(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st) {
+    static cudaError_t launch_group_w(const AttnArgs& a, int64_t blocks, size_t smem_bytes, cudaStream_t st,
+                                      bool copy_only = false) {
         if constexpr (sizeof(T) == 2 && !HM && !SEL) {
+            if constexpr (W == 4 && !APPEND) {
+                if (copy_only) {                        // (the measuring form: dsa_debug_copy_only)
+                    auto kern = dsa_attn_group_kernel<D, G, ST, 4, false, false, true>;
+                    const cudaError_t e = ensure_configured(kern, group_configured<4, false, ST, false, true>());
+                    if (e != cudaSuccess) return e;
+                    return launch_pdl(kern, (unsigned)blocks, 32 * 4, smem_bytes, st, a);
+                }
+            }
             if (W == 4 && a.early_list) {               // (the early-list form exists for four-warp blocks)
                 auto kern = dsa_attn_group_kernel<D, G, ST, 4, APPEND, true>;
                 const cudaError_t e = ensure_configured(kern, group_configured<4, APPEND, ST, true>());
@@ -162,16 +171,18 @@ struct KernelPick {
     }
     template <int ST>
     static cudaError_t launch_group_s(int w, bool append, const AttnArgs& a, int64_t blocks, size_t smem_bytes,
-                                      cudaStream_t st) {
+                                      cudaStream_t st, bool copy_only) {
+        if (copy_only && (w != 4 || append)) return cudaErrorInvalidValue;
         if (w == 4) return append ? launch_group_w<4, true, ST>(a, blocks, smem_bytes, st)
-                                  : launch_group_w<4, false, ST>(a, blocks, smem_bytes, st);
+                                  : launch_group_w<4, false, ST>(a, blocks, smem_bytes, st, copy_only);
         return append ? launch_group_w<2, true, ST>(a, blocks, smem_bytes, st)
                       : launch_group_w<2, false, ST>(a, blocks, smem_bytes, st);
     }
     static cudaError_t launch_group(int w, int stages, bool append, const AttnArgs& a, int64_t blocks,
-                                    size_t smem_bytes, cudaStream_t st) {
-        return stages == kGroupStagesShallow ? launch_group_s<kGroupStagesShallow>(w, append, a, blocks, smem_bytes, st)
-                                             : launch_group_s<kGroupStages>(w, append, a, blocks, smem_bytes, st);
+                                    size_t smem_bytes, cudaStream_t st, bool copy_only) {
+        return stages == kGroupStagesShallow
+                   ? launch_group_s<kGroupStagesShallow>(w, append, a, blocks, smem_bytes, st, copy_only)
+                   : launch_group_s<kGroupStages>(w, append, a, blocks, smem_bytes, st, copy_only);
     }
     // The same with tensor-map gather copies (four-warp blocks).
     static size_t smem_gather(int stages, int chunk, int bw) {
@@ -444,7 +455,7 @@ cudaError_t kernel_launch(const KernelQuery& q, bool append, const AttnArgs& a, 
         else if (q.mma && q.heads) err = P::launch_heads(append, a, blocks, smem, st);
         else if (q.mma && q.group_w > 0 && q.producers) err = P::launch_ws(q.group_stages, append, a, blocks, smem, st);
         else if (q.mma && q.group_w > 0 && q.gather) err = P::launch_gather(q.group_stages, append, a, maps, blocks, smem, st);
-        else if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st);
+        else if (q.mma && q.group_w > 0) err = P::launch_group(q.group_w, q.group_stages, append, a, blocks, smem, st, q.copy_only);
         else
         err = q.mma ? P::launch_mma(q.mma_warps, q.mma_kw, q.mma_stages, a, items, smem, st, append)
                     : P::launch(a, items, smem, st);

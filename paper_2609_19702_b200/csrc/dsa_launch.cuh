@@ -29,6 +29,7 @@ struct KernelQuery {
     int group_w;             // head-group tensor-core kernel: warps per block that share one row list for
                              // group_w x heads_per_warp kv heads (2 or 4); 0: not that kernel
     int group_stages;        // its ring depth: kGroupStages or kGroupStagesShallow
+    bool copy_only;          // head-group kernel (group_w 4, no fused step) in its measuring form: copies, no arithmetic
     bool gather;             // head-group kernel whose tiles are staged by tensor-map gather copies (group_w 4)
     bool producers;          // head-group kernel with a producer warp beside every consumer warp (group_w 4)
     bool heads;              // per-head-list tensor-core kernel (blocks of kHeadsWarps warps); sizes of its tables:

@@ -122,7 +122,29 @@ def random_valid_trace(rng: np.random.Generator, window: int, n_att: int, shape=
     return out.reshape(tuple(shape) + (max(m, 0),))
 
 
+_DRAWN: Dict[tuple, Dict[str, object]] = {}
+_DRAWN_BYTES = [0]
+_DRAWN_LIMIT = 3 << 30
+
+
 def make_inputs(w: Workload, seed: Optional[int] = None, poison: bool = True) -> Dict[str, object]:
+    """The batch of inputs for workload ``w`` (see _draw_inputs).  Drawing a few hundred million normal
+    variates takes seconds and the same (workload, seed) is asked for again and again, so batches are
+    kept per process (up to 3 GB) and every caller gets its own copy of the arrays."""
+    key = (w, seed, poison)
+    hit = _DRAWN.get(key)
+    if hit is None:
+        hit = _draw_inputs(w, seed, poison)
+        size = sum(v.nbytes for v in hit.values() if isinstance(v, np.ndarray))
+        if _DRAWN_BYTES[0] + size <= _DRAWN_LIMIT:
+            _DRAWN[key] = hit
+            _DRAWN_BYTES[0] += size
+        else:
+            return hit
+    return {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in hit.items()}
+
+
+def _draw_inputs(w: Workload, seed: Optional[int] = None, poison: bool = True) -> Dict[str, object]:
     """Draw one batch of inputs for workload ``w`` on the host.
 
     Returns a dict with

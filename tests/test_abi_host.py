@@ -192,6 +192,21 @@ def test_newer_entry_points_validate_before_touching_a_device(dsa):
     assert host_io(ctypes.byref(p), ctypes.byref(d), None, hp, hp, None, fake, fake, hp, hp, None, 0, None) == -1
 
 
+def test_copy_only_hook_refuses_plans_without_the_four_warp_head_group_kernel(dsa):
+    lib = ctypes.CDLL(dsa.LIB_PATH)
+    hook = lib.dsa_debug_copy_only
+    hook.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_size_t, ctypes.c_void_p]
+    fake = ctypes.c_void_p(0x50000)
+    d = _diag(dsa)
+    small = _problem(dsa, batch=8)                      # several warps per item: another kernel
+    assert hook(ctypes.byref(small), ctypes.byref(d), fake, fake, None, 0, None) == -2
+    f32 = _problem(dsa, batch=256, dtype=dsa.DSA_F32)   # CUDA cores
+    assert hook(ctypes.byref(f32), ctypes.byref(d), fake, fake, None, 0, None) == -2
+    bad = _problem(dsa, batch=256, head_dim=96)
+    assert hook(ctypes.byref(bad), ctypes.byref(d), fake, fake, None, 0, None) == -2
+    assert hook(None, ctypes.byref(d), fake, fake, None, 0, None) == -1
+
+
 def test_tensor_map_copies_only_on_request_and_only_with_a_2d_view(dsa):
     big = dict(batch=256, num_q_heads=32, num_kv_heads=32, max_seq_len=4360, max_prompt_len=200,
                stride_batch=4360 * 4096, stride_token=4096, stride_head=128)

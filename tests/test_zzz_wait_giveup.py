@@ -44,3 +44,38 @@ def test_a_wait_that_runs_out_is_counted_and_the_context_survives(dsa):
     ref = util.oracle_run(inp, ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride=w.stride)
     util.assert_close(out, lse, ref, what="after a give-up")
     assert dsa.dsa_wait_timeouts() == before + 1
+
+
+def test_copy_only_hook_runs_and_leaves_the_library_as_it_was(dsa):
+    """The measuring form of the head-group kernel: same plan, no arithmetic.  Its outputs mean nothing;
+    what is checked is that it runs, is not slower than the attention call it mirrors, and that the
+    attention call after it still matches the oracle."""
+    w = synth.workload(5, batch=32)
+    inp = synth.make_inputs(w)
+    prob = dsa.problem_from_host(inp)
+    diag = dsa.Diag(dsa.DSA_MASK_GRID, w.window, w.n_att, w.grid_w, w.row_extra)
+    plan = dsa.dsa_query_plan(prob, diag)
+    assert plan.block_warps == 4 and plan.per_head_lists == 0
+    out, lse = dsa.alloc_outputs(prob)
+    ws = dsa.alloc_workspace(prob, diag)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    t_copy = timed(lambda: dsa.dsa_debug_copy_only(prob, diag, out, lse, ws))
+    t_real = timed(lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws))
+    assert t_copy < 1.1 * t_real, "copy-only %.3f ms against %.3f ms with the arithmetic" % (t_copy, t_real)
+    ref = util.oracle_run(inp, ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride=w.stride, requests=[0, 7, 31])
+    util.assert_close(out[[0, 7, 31]], lse[[0, 7, 31]], ref, what="after the copy-only form")
+    small = dsa.problem_from_host(synth.make_inputs(synth.workload(5, batch=2)))
+    with pytest.raises(dsa.DsaError):
+        dsa.dsa_debug_copy_only(small, diag, *dsa.alloc_outputs(small))
+
