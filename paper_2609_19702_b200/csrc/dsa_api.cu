@@ -228,7 +228,7 @@ int choose_heads_per_warp(const dsa_problem* p, const Plan& pl, int w, int64_t b
             const double load = std::min(waves, 1.0) * full;
             const double per_tile = load <= 1.0 ? 0.67 + 0.33 * load : 1.0 + 1.1 * (load - 1.0);
             double cost = block_time * per_tile;
-            if (waves > 1.0) cost *= waves * (1.0 + 0.5 * std::max(0.0, std::ceil(waves - 0.05) / waves - 1.0));
+            if (waves > 1.0) cost *= waves * (1.0 + 0.5 * std::max(0.0, std::ceil(waves - 0.004) / waves - 1.0));
             if (shallow) cost *= 1.02;
             if (best == 0 || cost < best_cost * 1.005) {    // (ties go to the larger U: a grid that just fits has no turnover)
                 best = u; best_cost = cost;

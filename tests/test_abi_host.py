@@ -255,6 +255,22 @@ def test_producer_warps_only_for_grids_of_more_than_one_wave(dsa):
     assert plan(256, dsa.plan_group(2, 1) | dsa.DSA_PLAN_PRODUCERS).producer_warps == 0
 
 
+def test_no_plan_spills_a_few_blocks_into_a_second_wave(dsa):
+    """304 deep-ring blocks on 296 slots ran 21 % slower than a plan that fits (batch 152; batch 232 likewise
+    with the shallow ring): the estimate must not round such a spill away."""
+    shape = dict(num_q_heads=32, num_kv_heads=32, max_seq_len=4360, max_prompt_len=200,
+                 stride_batch=4360 * 4096, stride_token=4096, stride_head=128)
+    diag = _diag(dsa, window=512, n_att=208, grid_w=64)
+    for batch in range(8, 264, 4):
+        rc, info = _plan(dsa, _problem(dsa, batch=batch, **shape), diag)
+        assert rc == 0
+        if info.heads_per_block == 0:
+            continue
+        slots = 148 * (2 if info.stages == 3 else 3)
+        waves = info.grid_blocks / slots
+        assert not 1.0 < waves < 1.1, (batch, info.grid_blocks, info.stages)
+
+
 def test_ring_depth_follows_the_wave_estimate(dsa):
     def stages(batch):
         rc, info = _plan(dsa, _problem(dsa, batch=batch, num_q_heads=32, num_kv_heads=32, max_seq_len=4360,
