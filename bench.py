@@ -462,8 +462,10 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
             out, lse = dsa.alloc_outputs(prob)
             ldiag = diag
             if kind == "sparse_select":
+                # the lists and their bitmap form (dsa_diag_params.skip_bitmap), both grown by the selection
                 trace = torch.zeros((b, h, 512 - 52), dtype=torch.int32, device=dev)
-                ldiag = dsa.Diag(dsa.DSA_MASK_LIST, 512, 52, skip_offsets=trace, select=True)
+                bitmap = torch.zeros((b, h, 512 // 32), dtype=torch.int32, device=dev)
+                ldiag = dsa.Diag(dsa.DSA_MASK_LIST, 512, 52, skip_offsets=trace, select=True, skip_bitmap=bitmap)
             layers.append((prob, out, lse, dsa.alloc_workspace(prob, ldiag), ldiag))
 
         def step():
@@ -480,8 +482,11 @@ def decode_loop_bench(torch, dsa, synth, dev, n_layers=8, batch=16,
                 dsa.dsa_advance_seq_len(shared_seq, s_max)
 
         def reset(value):
-            for prob, _, _, _, _ in layers:
+            for prob, _, _, _, ldiag in layers:
                 prob.seq_len.fill_(value)
+                if value == l_p and ldiag is not None and ldiag.skip_bitmap is not None:
+                    ldiag.skip_offsets.zero_()             # the image starts over: empty lists, empty bitmaps
+                    ldiag.skip_bitmap.zero_()
 
         step()                                             # eager warm-up (one-time kernel set-up)
         torch.cuda.synchronize()

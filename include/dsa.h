@@ -209,6 +209,15 @@ typedef struct dsa_diag_params {
     int32_t trace_len;            /* LIST: entries per trace, >= window - n_att                    */
     int32_t n_sink;               /* first decode tokens always kept (>= 0; 0 = none)              */
     int32_t select;               /* LIST, mask_heads == H_q: also run the phase-2 selection       */
+    uint32_t *skip_bitmap;        /* LIST, optional (NULL: none): device [B, mask_heads, ceil(window / 32)]  */
+                                  /* words; bit o of a head's row is set iff distance o is one of its        */
+                                  /* ACTIVE skip_offsets entries (the first n_act).  The same information    */
+                                  /* as the list, in the form the per-head-list kernel wants: it then reads  */
+                                  /* window / 8 bytes per head instead of scattering the list into a bitmap  */
+                                  /* itself.  dsa_build_skip_bitmap() fills it from skip_offsets; calls with */
+                                  /* `select` keep it up to date (they set the bit of every entry they       */
+                                  /* write).  The caller clears it together with the list when a request     */
+                                  /* starts over.  Kernels other than the per-head-list one read the list.   */
 } dsa_diag_params;
 
 /* What a call will launch (filled by dsa_query_plan; for reporting and for tests). */
@@ -257,6 +266,10 @@ DSA_API int32_t dsa_wait_timeouts(int32_t *count_out);
  * kernel (dsa_plan_info.block_warps == 4, per_head_lists == 0).  Arguments as dsa_decode_attention_sparse. */
 DSA_API int32_t dsa_debug_copy_only(const dsa_problem *problem, const dsa_diag_params *diag, void *out, float *lse,
                                     void *workspace, size_t workspace_bytes, void *stream);
+/* Fills diag->skip_bitmap from diag->skip_offsets for the requests' current seq_len: row (b, mask head)
+ * gets the bits of that head's first n_act entries that lie in [0, window), all other bits are cleared.
+ * LIST mode only; both pointers required.  Asynchronous on `stream`. */
+DSA_API int32_t dsa_build_skip_bitmap(const dsa_problem *problem, const dsa_diag_params *diag, void *stream);
 /* Test hook for that mechanism: launches one warp on `stream` that waits, with the same bound, on an
  * mbarrier nothing ever arrives on.  The wait runs out after about a second, the counter above goes
  * up by one, the kernel ends and the context stays usable.  Asynchronous like every launch. */

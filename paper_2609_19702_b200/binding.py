@@ -40,7 +40,7 @@ EXPORTS = ["dsa_version", "dsa_status_string", "dsa_last_cuda_error", "dsa_works
            "dsa_combine_splits", "dsa_debug_kept_indices",
            "dsa_decode_attention_static_scratch", "dsa_append_kv", "dsa_decode_attention_host_io",
            "dsa_decode_attention_host_mapped", "dsa_decode_step", "dsa_advance_seq_len", "dsa_prepare",
-           "dsa_wait_timeouts", "dsa_debug_wait_giveup", "dsa_debug_copy_only"]
+           "dsa_wait_timeouts", "dsa_debug_wait_giveup", "dsa_debug_copy_only", "dsa_build_skip_bitmap"]
 
 
 class dsa_problem(ctypes.Structure):
@@ -64,7 +64,7 @@ class dsa_diag_params(ctypes.Structure):
                 ("grid_w", ctypes.c_int32), ("row_extra", ctypes.c_int32),
                 ("skip_offsets", ctypes.c_void_p), ("mask_heads", ctypes.c_int32),
                 ("trace_len", ctypes.c_int32), ("n_sink", ctypes.c_int32),
-                ("select", ctypes.c_int32)]
+                ("select", ctypes.c_int32), ("skip_bitmap", ctypes.c_void_p)]
 
 
 class dsa_plan_info(ctypes.Structure):
@@ -106,6 +106,8 @@ def _load() -> ctypes.CDLL:
     lib.dsa_wait_timeouts.argtypes = [ctypes.POINTER(i32)]
     lib.dsa_debug_copy_only.restype = i32
     lib.dsa_debug_copy_only.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.dsa_build_skip_bitmap.restype = i32
+    lib.dsa_build_skip_bitmap.argtypes = [vp, vp, vp]
     lib.dsa_debug_wait_giveup.restype = i32
     lib.dsa_debug_wait_giveup.argtypes = [vp]
     lib.dsa_prepare.restype = i32
@@ -215,6 +217,7 @@ class Diag:
     skip_offsets: Optional[torch.Tensor] = None   # int32 [B, mask_heads, trace_len] (LIST)
     n_sink: int = 0
     select: bool = False                          # LIST: also append the next trace entry (in place)
+    skip_bitmap: Optional[torch.Tensor] = None    # int32 [B, mask_heads, ceil(window / 32)]: the lists as bits
 
     def c_struct(self) -> dsa_diag_params:
         d = dsa_diag_params()
@@ -227,6 +230,11 @@ class Diag:
             assert t.dtype == torch.int32 and t.is_contiguous() and t.dim() == 3
             d.skip_offsets = t.data_ptr()
             d.mask_heads, d.trace_len = t.shape[1], t.shape[2]
+        if self.skip_bitmap is not None:
+            bm = self.skip_bitmap
+            assert self.skip_offsets is not None and bm.dtype == torch.int32 and bm.is_contiguous()
+            assert tuple(bm.shape) == (self.skip_offsets.shape[0], self.skip_offsets.shape[1], (self.window + 31) // 32)
+            d.skip_bitmap = bm.data_ptr()
         return d
 
 
@@ -257,6 +265,12 @@ def dsa_wait_timeouts() -> int:
     n = ctypes.c_int32(0)
     _check("dsa_wait_timeouts", _lib.dsa_wait_timeouts(ctypes.byref(n)))
     return int(n.value)
+
+
+def dsa_build_skip_bitmap(problem: Problem, diag: Diag, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Fill diag.skip_bitmap from diag.skip_offsets for the requests' current seq_len."""
+    p, d = problem.c_struct(), diag.c_struct()
+    _check("dsa_build_skip_bitmap", _lib.dsa_build_skip_bitmap(_ref(p), _ref(d), _stream(stream)))
 
 
 def dsa_debug_wait_giveup(stream: Optional[torch.cuda.Stream] = None) -> None:

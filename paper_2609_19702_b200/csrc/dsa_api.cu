@@ -158,6 +158,7 @@ int32_t check_diag(const dsa_problem* p, const dsa_diag_params* d) {
         return DSA_ERR_INVALID_ARG;
     if (d->trace_len < d->window - d->n_att) return DSA_ERR_INVALID_ARG;
     if (d->window - d->n_att > 0 && p->batch > 0 && !d->skip_offsets) return DSA_ERR_INVALID_ARG;
+    if (d->skip_bitmap && (reinterpret_cast<uintptr_t>(d->skip_bitmap) & 3u)) return DSA_ERR_INVALID_ARG;
     if (d->select && d->mask_heads != p->num_q_heads) return DSA_ERR_UNSUPPORTED;   // one selection per attention head
     if (d->select && d->n_sink >= d->n_att) return DSA_ERR_INVALID_ARG;             // no candidate would be left
     return DSA_OK;
@@ -557,6 +558,7 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
     a->mask.mask_heads = (d && pl.mode == MODE_LIST) ? d->mask_heads : 1;
     a->mask.trace_len = (d && pl.mode == MODE_LIST) ? d->trace_len : 0;
     a->mask.bitmap_words = pl.bitmap_words;
+    a->mask.skip_bitmap = (d && pl.mode == MODE_LIST) ? d->skip_bitmap : nullptr;
     a->chunk = pl.chunk; a->n_split = pl.n_split;
     a->heads_per_warp = pl.group_u;
     a->dir_cap = pl.dir_cap; a->kidx_cap = pl.kidx_cap;
@@ -577,7 +579,8 @@ void fill_args(const dsa_problem* p, const dsa_diag_params* d, const Plan& pl, A
 template <typename T>
 cudaError_t launch_combine_t(const float* out_part, const float* lse_part, int64_t rows, int D, int n_split,
                              void* out, float* lse, cudaStream_t st, const float* sel_val, const int* sel_off,
-                             const int* sel_k, int* trace, int trace_len, bool after_attention) {
+                             const int* sel_k, int* trace, int trace_len, bool after_attention,
+                             unsigned* skip_bitmap, int bitmap_words, int window) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)rows);
     cfg.blockDim = dim3((unsigned)((D + 31) / 32 * 32));    // whole warps: the block reductions shuffle with a full mask
@@ -589,20 +592,22 @@ cudaError_t launch_combine_t(const float* out_part, const float* lse_part, int64
     cfg.attrs = attr;
     cfg.numAttrs = after_attention ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, dsa_combine_kernel<T>, out_part, lse_part, D, n_split, out, lse, sel_val,
-                              sel_off, sel_k, trace, trace_len);
+                              sel_off, sel_k, trace, trace_len, skip_bitmap, bitmap_words, window);
 }
 
 int32_t launch_combine(const float* out_part, const float* lse_part, int64_t rows, int D, int n_split,
                        void* out, float* lse, int dtype, cudaStream_t st, const float* sel_val = nullptr,
                        const int* sel_off = nullptr, const int* sel_k = nullptr, int* trace = nullptr,
-                       int trace_len = 0, bool after_attention = false) {
+                       int trace_len = 0, bool after_attention = false, unsigned* skip_bitmap = nullptr,
+                       int bitmap_words = 0, int window = 0) {
     if (rows == 0) return DSA_OK;
     const cudaError_t e =
         dtype == DSA_BF16
             ? launch_combine_t<__nv_bfloat16>(out_part, lse_part, rows, D, n_split, out, lse, st, sel_val, sel_off,
-                                              sel_k, trace, trace_len, after_attention)
+                                              sel_k, trace, trace_len, after_attention, skip_bitmap, bitmap_words,
+                                              window)
             : launch_combine_t<float>(out_part, lse_part, rows, D, n_split, out, lse, st, sel_val, sel_off, sel_k,
-                                      trace, trace_len, after_attention);
+                                      trace, trace_len, after_attention, skip_bitmap, bitmap_words, window);
     return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
@@ -741,7 +746,8 @@ int32_t run_attention(const dsa_problem* p, const dsa_diag_params* d, void* out,
     if (pl.n_split > 1)
         return launch_combine(a.out_part, a.lse_part, (int64_t)p->batch * p->num_q_heads, p->head_dim,
                               pl.n_split, out, lse, p->dtype, st, a.sel_val_part, a.sel_off_part, a.sel_k,
-                              pl.select ? d->skip_offsets : nullptr, pl.select ? d->trace_len : 0, true);
+                              pl.select ? d->skip_offsets : nullptr, pl.select ? d->trace_len : 0, true,
+                              pl.select ? d->skip_bitmap : nullptr, pl.bitmap_words, pl.select ? d->window : 0);
     return DSA_OK;
 }
 
@@ -788,6 +794,21 @@ int32_t dsa_last_cuda_error(void) { return g_last_cuda_error; }
 int32_t dsa_debug_copy_only(const dsa_problem* problem, const dsa_diag_params* diag, void* out, float* lse,
                             void* workspace, size_t workspace_bytes, void* stream) {
     return run_attention(problem, diag, out, lse, workspace, workspace_bytes, stream, nullptr, nullptr, true);
+}
+
+int32_t dsa_build_skip_bitmap(const dsa_problem* problem, const dsa_diag_params* diag, void* stream) {
+    if (!diag) return DSA_ERR_INVALID_ARG;
+    Plan pl;
+    const int32_t rc = make_plan(problem, diag, &pl);
+    if (rc != DSA_OK) return rc;
+    if (pl.mode != MODE_LIST || !diag->skip_bitmap) return DSA_ERR_INVALID_ARG;
+    if (problem->batch == 0) return DSA_OK;
+    AttnArgs a;
+    fill_args(problem, diag, pl, &a);
+    dsa_build_skip_bitmap_kernel<<<(unsigned)(problem->batch * diag->mask_heads), 128, 0,
+                                   reinterpret_cast<cudaStream_t>(stream)>>>(a);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DSA_OK : cuda_fail(e);
 }
 
 int32_t dsa_debug_wait_giveup(void* stream) {

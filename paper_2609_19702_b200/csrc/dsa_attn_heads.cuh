@@ -141,7 +141,22 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
         const int mh = a.mask.mask_heads == 1 ? 0 : (a.mask.mask_heads == a.H_kv ? kvh : h);
         return a.mask.skip_offsets + ((int64_t)b * a.mask.mask_heads + mh) * a.mask.trace_len;
     };
+    // the same head's row of the caller's bitmap form of the lists (MaskArgs::skip_bitmap), if there is one
+    auto bitmap_of = [&](int kvh, int s) {
+        const int h = kvh * G + s;
+        const int mh = a.mask.mask_heads == 1 ? 0 : (a.mask.mask_heads == a.H_kv ? kvh : h);
+        return a.mask.skip_bitmap + ((int64_t)b * a.mask.mask_heads + mh) * a.mask.bitmap_words;
+    };
     auto prefetch_trace = [&](int kvh, int (&pre)[PRE]) {
+        if (a.mask.skip_bitmap) {                       // (then the words of the bitmap travel instead of list entries)
+            const unsigned* src = bitmap_of(kvh, 0);
+#pragma unroll
+            for (int k = 0; k < PRE; ++k) {
+                const int i = k * 32 + lane;
+                pre[k] = (!m.keep_all && i < a.mask.bitmap_words) ? (int)src[i] : 0;
+            }
+            return;
+        }
         const int* trace = trace_of(kvh, 0);
 #pragma unroll
         for (int k = 0; k < PRE; ++k) {
@@ -153,7 +168,30 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
         unsigned short* kidx = kidx_of(buf);
         unsigned char* hbits = hbits_of(buf);
         __syncwarp();
-        if (!m.keep_all) {
+        if (!m.keep_all && a.mask.skip_bitmap) {
+            // The caller keeps the lists as bitmaps, 32 distances per word: split every word into the two
+            // 16-distance words of the layout used here.  Nothing to scatter, no atomics.
+#pragma unroll
+            for (int s = 0; s < C::SLOTS; ++s) {
+                const unsigned* src = bitmap_of(kvh, s);
+                for (int i0 = 0; i0 < a.mask.bitmap_words; i0 += 32) {
+                    const int i = i0 + lane;
+                    if (i < a.mask.bitmap_words) {
+                        unsigned wd = 0u;
+                        bool have = false;
+                        if (s == 0) {
+#pragma unroll
+                            for (int k = 0; k < PRE; ++k)
+                                if (i0 == k * 32) { wd = (unsigned)pre[k]; have = true; }
+                        }
+                        if (!have) wd = src[i];
+                        bitmaps[s * words + 2 * i] = wd & 0xffffu;
+                        bitmaps[s * words + 2 * i + 1] = wd >> 16;
+                    }
+                }
+            }
+            __syncwarp();
+        } else if (!m.keep_all) {
             for (int i = lane; i < C::SLOTS * words; i += 32) bitmaps[i] = 0u;
             __syncwarp();
             auto mark = [&](int s, int o) {
@@ -487,7 +525,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
                             a.sel_off_part[row * a.n_split + split] = off;
                             a.sel_k[row] = m.sel_k;
                         } else if (m.sel_k >= 0) {
-                            a.mask.skip_offsets[row * a.mask.trace_len + m.sel_k] = off;
+                            record_selection(a.mask, row, m.sel_k, off);
                         }
                     }
                 }

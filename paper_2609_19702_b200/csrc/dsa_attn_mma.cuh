@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(32 * W * KW) dsa_attn_mma_kernel(const AttnArg
                         a.sel_off_part[row * a.n_split + split] = off;
                         a.sel_k[row] = m.sel_k;
                     } else if (m.sel_k >= 0) {
-                        a.mask.skip_offsets[row * a.mask.trace_len + m.sel_k] = off;
+                        record_selection(a.mask, row, m.sel_k, off);
                     }
                 }
             }

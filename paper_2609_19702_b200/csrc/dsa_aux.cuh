@@ -15,7 +15,8 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
                                    const float* __restrict__ sel_val_part = nullptr,
                                    const int* __restrict__ sel_off_part = nullptr,
                                    const int* __restrict__ sel_k = nullptr, int* trace = nullptr,
-                                   int trace_len = 0) {
+                                   int trace_len = 0, unsigned* skip_bitmap = nullptr, int bitmap_words = 0,
+                                   int window = 0) {
     // launched behind an attention kernel with programmatic serialisation: wait for that grid
     // and its writes (returns at once after an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -78,6 +79,8 @@ __global__ void dsa_combine_kernel(const float* __restrict__ out_part, const flo
                 if (o >= 0 && (v < bv || (v == bv && o > bo))) { bv = v; bo = o; }
             }
             trace[row * trace_len + k] = bo;
+            if (skip_bitmap && bo >= 0 && bo < window)         // (the caller's bitmap form of the list, kept in step)
+                atomicOr(&skip_bitmap[row * bitmap_words + (bo >> 5)], 1u << (bo & 31));
         }
     }
 }
@@ -110,6 +113,22 @@ __global__ void dsa_append_kv_kernel(const AttnArgs a, const T* __restrict__ k_n
     }
     __syncthreads();                                       // every thread has read S
     if (advance && threadIdx.x == 0) a.seq_len_rw[b] = S + 1;
+}
+
+// ---- the bitmap form of the skip lists (dsa_build_skip_bitmap): one block per (request, mask head) sets
+// the bits of the head's first n_act entries and clears the rest of its row
+__global__ void dsa_build_skip_bitmap_kernel(const AttnArgs a) {
+    const int b = blockIdx.x / a.mask.mask_heads;
+    const ReqMask m = req_mask_setup(a.mask, a.seq_len[b], req_prompt_len(a, b), a.max_seq_len);
+    unsigned* row = a.mask.skip_bitmap + (int64_t)blockIdx.x * a.mask.bitmap_words;
+    const int* trace = a.mask.skip_offsets + (int64_t)blockIdx.x * a.mask.trace_len;
+    for (int i = threadIdx.x; i < a.mask.bitmap_words; i += blockDim.x) row[i] = 0u;
+    __syncthreads();
+    const int n_act = m.keep_all ? 0 : m.n_act;
+    for (int i = threadIdx.x; i < n_act; i += blockDim.x) {
+        const int o = trace[i];
+        if (o >= 0 && o < a.mask.window) atomicOr(&row[o >> 5], 1u << (o & 31));
+    }
 }
 
 // One warp waits, bounded, on an mbarrier that nobody ever arrives on: the wait runs out, the warp

@@ -28,7 +28,16 @@ struct MaskArgs {
     int mask_heads;
     int trace_len;
     int bitmap_words;          // 32-bit words per LIST bitmap = ceil(window / 32)
+    unsigned* skip_bitmap;     // [B, mask_heads, bitmap_words] or NULL: the active entries of skip_offsets as bits
 };
+
+// The selection's result for trace slot k of mask row `row` (b * mask_heads + head): the list entry and,
+// where the caller keeps one, the bit of the bitmap.
+__device__ __forceinline__ void record_selection(const MaskArgs& a, int64_t row, int k, int off) {
+    a.skip_offsets[row * a.trace_len + k] = off;
+    if (a.skip_bitmap && off >= 0 && off < a.window)
+        atomicOr(&a.skip_bitmap[row * a.bitmap_words + (off >> 5)], 1u << (off & 31));
+}
 
 // Per-request constants of the mask.
 struct ReqMask {

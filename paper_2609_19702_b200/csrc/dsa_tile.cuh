@@ -320,7 +320,7 @@ struct ItemState {
                     a.sel_off_part[row * a.n_split + split] = off;
                     a.sel_k[row] = m.sel_k;
                 } else if (m.sel_k >= 0) {
-                    a.mask.skip_offsets[row * a.mask.trace_len + m.sel_k] = off;
+                    record_selection(a.mask, row, m.sel_k, off);
                 }
             }
         }
