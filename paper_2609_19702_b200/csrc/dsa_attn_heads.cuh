@@ -379,7 +379,11 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
     const int hc = (lane & 3) * 2, kr = lane >> 2;
     const int lm_row_k = (lane & 7) + ((lane >> 3) & 1) * 8, lm_chk_k = lane >> 4;
     const int lm_row_v = (lane & 7) + (lane >> 4) * 8, lm_chk_v = (lane >> 3) & 1;
-    const int cand_lo = m.L_p + a.mask.n_sink;
+    // Selection candidates are the kept decode keys that are no sinks.  Kept rows ascend in position, the
+    // always-kept rows come first and the sinks still inside the window are the first window rows (all
+    // kept), so "candidate" is a threshold on the row's rank, and the oldest of equal logits is the lowest
+    // rank: the tile loop tracks ranks and only the winner is turned into a position.
+    const int cand_row = prefix + min(max(0, m.L_p + a.mask.n_sink - m.w_lo), n_win);
     int cslot = 0;
 
 #pragma unroll 1
@@ -435,11 +439,7 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
                 bits0 = v0 ? (g0 < 0 ? ALL : (unsigned)hbits[g0]) : 0u;
                 bits1 = v1 ? (g1 < 0 ? ALL : (unsigned)hbits[g1]) : 0u;
             }
-            int pos0 = 0, pos1 = 0;
-            if (SELECT) {
-                pos0 = v0 ? (g0 < 0 ? r_lo + r0 : m.w_lo + (int)kidx[g0]) : 0;
-                pos1 = v1 ? (g1 < 0 ? r_lo + r1 : m.w_lo + (int)kidx[g1]) : 0;
-            }
+            const int pos0 = r_lo + r0, pos1 = r_lo + r1;      // (ranks; see cand_row)
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const bool on0 = v0 && (!HEADMASK || ((bits0 >> (hc + j)) & 1u));
@@ -448,8 +448,8 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
                 float x1 = on1 ? s[2 + j] * a.scale_log2 : -INFINITY;
                 if (SELECT) {
                     // keys arrive in ascending position: a strict "<" keeps the oldest of equal logits
-                    if (on0 && pos0 >= cand_lo && x0 < bestv[j]) { bestv[j] = x0; bestp[j] = pos0; }
-                    if (on1 && pos1 >= cand_lo && x1 < bestv[j]) { bestv[j] = x1; bestp[j] = pos1; }
+                    if (on0 && pos0 >= cand_row && x0 < bestv[j]) { bestv[j] = x0; bestp[j] = pos0; }
+                    if (on1 && pos1 >= cand_row && x1 < bestv[j]) { bestv[j] = x1; bestp[j] = pos1; }
                 }
                 float mx = fmaxf(x0, x1);
                 mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 4));
@@ -519,7 +519,8 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
                     if (a.n_split > 1) a.lse_part[row * a.n_split + split] = lse;
                     else a.lse[row] = lse;
                     if (SELECT) {
-                        const int off = bp == 0x7fffffff ? -1 : (m.S - 1) - bp;
+                        // (rank -> position: a candidate is a window row)
+                        const int off = bp == 0x7fffffff ? -1 : (m.S - 1) - (m.w_lo + (int)kidx[bp - prefix]);
                         if (a.n_split > 1) {
                             a.sel_val_part[row * a.n_split + split] = bv;
                             a.sel_off_part[row * a.n_split + split] = off;
