@@ -206,7 +206,9 @@ def algorithmic_bytes(w, host, mode, blocks_touched, list_mask=None):
     keys for the sparse call (the attended count of Algorithm 1), p for the dense call.
     list_mask (LIST masks): {"mask_heads": 1 | H_kv | H_q, "union_rows": total rows over
     (request, kv head) when query heads of a group keep different rows, else None}; adds the
-    trace entries every mask head reads, mask_heads x n_act x 4 bytes per request."""
+    trace entries every mask head reads, mask_heads x n_act x 4 bytes per request -- or, with
+    "bitmap_words" (the lists given as bitmaps, dsa_diag_params.skip_bitmap), the bitmap rows read instead:
+    mask_heads x bitmap_words x 4 bytes per request."""
     esize = 2
     p = host["position"].astype(np.int64)
     lp = host["prompt_len"].astype(np.int64)
@@ -217,7 +219,10 @@ def algorithmic_bytes(w, host, mode, blocks_touched, list_mask=None):
     if list_mask is not None:
         if list_mask.get("union_rows") is not None:
             kv_rows = int(list_mask["union_rows"])
-        trace = 4 * int(list_mask["mask_heads"]) * int(list_active_entries(p, w.window, w.n_att).sum())
+        if list_mask.get("bitmap_words"):
+            trace = 4 * int(list_mask["mask_heads"]) * int(list_mask["bitmap_words"]) * len(p)
+        else:
+            trace = 4 * int(list_mask["mask_heads"]) * int(list_active_entries(p, w.window, w.n_att).sum())
     kv = kv_rows * w.head_dim * esize * 2
     qo = w.batch * w.num_q_heads * (2 * w.head_dim * esize + 4)
     table = 4 * int(blocks_touched)
@@ -706,11 +711,16 @@ def run_ours(args):
         trace = torch.from_numpy(np.ascontiguousarray(
             few[lrng.integers(0, 8, size=(w.batch, w.num_q_heads))])).to(dev)
         group = w.num_q_heads // w.num_kv_heads
-        for key, sel in (("list_per_head", False), ("list_per_head_select", True)):
-            ldiag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=trace, select=sel)
+        words = (w.window + 31) // 32
+        bitmap = torch.zeros((w.batch, w.num_q_heads, words), dtype=torch.int32, device=dev)
+        for key, sel, bm in (("list_per_head", False, None), ("list_per_head_select", True, None),
+                             ("list_per_head_bitmap", False, bitmap), ("list_per_head_bitmap_select", True, bitmap)):
+            ldiag = dsa.Diag(dsa.DSA_MASK_LIST, w.window, w.n_att, skip_offsets=trace, select=sel, skip_bitmap=bm)
+            if bm is not None:
+                dsa.dsa_build_skip_bitmap(prob, ldiag)      # (the lists as they stand now, as bits)
             lws = dsa.alloc_workspace(prob, ldiag)
             lplan = dsa.dsa_query_plan(prob, ldiag)
-            lmask = {"mask_heads": w.num_q_heads, "union_rows": None}
+            lmask = {"mask_heads": w.num_q_heads, "union_rows": None, "bitmap_words": words if bm is not None else 0}
             if group > 1:
                 lidx, lcnt = dsa.dsa_debug_kept_indices(prob, ldiag, inputs["max_seq_len"])
                 lmask["union_rows"] = union_rows(lidx.cpu().numpy(), lcnt.cpu().numpy(), group)
