@@ -144,7 +144,8 @@ typedef struct dsa_problem {
 #define DSA_PLAN_PRODUCERS     0x100000u /* head-group kernel, 4 warps: a producer warp beside every consumer warp */
 #define DSA_PLAN_NO_PRODUCERS  0x200000u /* never                                                       */
 /* Not a planner switch but a promise about the stream: no launch that can still be running when this
- * call's kernel starts writes seq_len, prompt_len, block_table or the skip lists.  The attention kernels
+ * call's kernel starts writes seq_len, prompt_len, block_table or the skip lists (skip_offsets and
+ * skip_bitmap; a call with `select` writes both, for its own layer).  The attention kernels
  * chain with programmatic dependent launch and let their successor start before they have waited for
  * their own predecessor, so "still running" means: the launch just before this call and, if that is an
  * attention call of this library, the launches before it in turn, back to the first launch that does
