@@ -48,7 +48,7 @@
 extern "C" {
 #endif
 
-#define DSA_VERSION 100
+#define DSA_VERSION 101  /* 101: dsa_problem.plan_flags promise bit, dsa_diag_params.skip_bitmap, dsa_plan_info grew */
 
 /* exported symbols (the library is built with hidden visibility for everything else) */
 #if defined(__GNUC__)

@@ -44,7 +44,7 @@ def test_wait_timeouts_validates_its_argument(dsa):
 
 
 def test_version_and_status_strings(dsa):
-    assert dsa.dsa_version() == 100
+    assert dsa.dsa_version() == 101
     lib = ctypes.CDLL(dsa.LIB_PATH)
     lib.dsa_status_string.restype = ctypes.c_char_p
     assert lib.dsa_status_string(0) == b"ok"
