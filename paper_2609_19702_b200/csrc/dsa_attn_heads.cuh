@@ -11,7 +11,8 @@
 // head's skip trace without touching global memory again: the trace goes into a bitmap over window
 // distances (16 distances per 32-bit word, so that the shared-memory atomics of a warp spread over
 // twice as many words), and the kept candidates are enumerated 16 distances per lane (mask,
-// popcount, one suffix scan across the warp, a handful of stores) into
+// popcount, one suffix scan across the warp, a handful of stores; where the caller also keeps the lists
+// as bitmaps, MaskArgs::skip_bitmap, the head's row is copied instead of scattered) into
 //   kidx[j]     candidate index of the j-th kept window row, ascending   (16 bits per row)
 //   hbits[j]    which query heads of the group keep it                   (grouped queries only)
 // Every warp streams U heads back to back through one ring that never drains in between: while the
@@ -390,7 +391,10 @@ __global__ void __launch_bounds__(32 * W) dsa_attn_heads_kernel(const AttnArgs a
     for (int u = 0; u < U; ++u) {
         const int kvh = kvh0 + u * W;
         cur_kvh = kvh;
-        // the ring holds the first tiles of this head: work out the next head's rows while they fly
+        // the ring holds the first tiles of this head: work out the next head's rows while they fly.  No
+        // tile is being consumed meanwhile, so the slot the last head's last tile has just left can fly too.
+        nxt_valid = false;                              // (nothing of the next head is known yet)
+        if (u + 1 < U) { while (inflight < STAGES && try_issue()) {} }
         nxt_valid = u + 1 < U;
         if (nxt_valid) {
             nxt_kvh = kvh + W;
