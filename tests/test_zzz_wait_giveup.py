@@ -72,7 +72,7 @@ def test_copy_only_hook_runs_and_leaves_the_library_as_it_was(dsa):
 
     t_copy = timed(lambda: dsa.dsa_debug_copy_only(prob, diag, out, lse, ws))
     t_real = timed(lambda: dsa.dsa_decode_attention_sparse(prob, diag, out, lse, ws))
-    assert t_copy < 1.1 * t_real, "copy-only %.3f ms against %.3f ms with the arithmetic" % (t_copy, t_real)
+    assert t_copy < 1.25 * t_real, "copy-only %.3f ms against %.3f ms with the arithmetic" % (t_copy, t_real)
     ref = util.oracle_run(inp, ora.MODE_GRID, n_r=w.window, n_att=w.n_att, stride=w.stride, requests=[0, 7, 31])
     util.assert_close(out[[0, 7, 31]], lse[[0, 7, 31]], ref, what="after the copy-only form")
     small = dsa.problem_from_host(synth.make_inputs(synth.workload(5, batch=2)))
